@@ -1,0 +1,153 @@
+/*
+ * mxattn — MXFP4 attention forward with Universal Optimal Scaling (UOS) and Pre-Normalization
+ * Quantization (PNQ) for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     The library allocates no memory, never frees, and (except where stated) never
+ *     synchronizes: work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).
+ *   - Every device pointer must be 16-byte aligned.
+ *   - Return value: MXATTN_OK (0) or a negative mxattn_status.  On an argument error nothing
+ *     is launched.  Inputs must be finite; NaN/Inf give unspecified values but never a hang.
+ *   - bf16 tensors are contiguous, row-major, innermost dimension last.
+ *
+ * Number formats (paper, Section 2 "MXFP4 Block Quantization")
+ *   - A block is 32 consecutive elements along the block axis that share one scale
+ *     sigma = 2^e, stored as an E8M0 byte e + 127 (0xFF is never produced).
+ *   - Elements are E2M1 codes: bit 3 = sign, bits 0-2 = index into {0, .5, 1, 1.5, 2, 3, 4, 6};
+ *     round-to-nearest (ties to the even code), saturating at 6.  The sign of the input is kept
+ *     even when the magnitude rounds to zero.
+ *   - Codes are packed two per byte along the block axis: element 2k in bits 0-3 of byte k,
+ *     element 2k+1 in bits 4-7.
+ */
+#ifndef MXATTN_H
+#define MXATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Shared-scale rule.
+ * OCP: e = floor(log2 M) - 2 (paper Eq. 5, the floor rule; normalized block maximum in [4, 8)).
+ * UOS: e = ceil(log2(M / 7.25)) (paper Eq. 13 with q* = 29/4, Theorem 1, Algorithm 1;
+ *      normalized block maximum in (3.625, 7.25]).
+ * M is the largest magnitude in the block; an all-zero block gets sigma = 1 (byte 127) and
+ * all-zero codes; e is clamped to [-127, 127]. */
+typedef enum { MXATTN_MODE_OCP = 0, MXATTN_MODE_UOS = 1 } mxattn_mode;
+
+/* Flags of the forward pass.
+ * UOS      : use the UOS rule for Q, K, V and the softmax tiles (else the OCP rule for all four).
+ * PNQ      : the row sum l is accumulated from the QUANTIZED exponentials (paper Eq. 22,
+ *            Algorithm 2 line 14); without it l is accumulated from the unquantized ones
+ *            (the "direct" placement, paper Eq. 12).
+ * OUT_FP32 : `o` is fp32 instead of bf16. */
+enum { MXATTN_FLAG_UOS = 1, MXATTN_FLAG_PNQ = 2, MXATTN_FLAG_OUT_FP32 = 4 };
+
+typedef enum {
+  MXATTN_OK = 0,
+  MXATTN_EINVAL = -1,       /* null pointer, non-positive size, unknown mode / flag / layout */
+  MXATTN_EUNSUPPORTED = -2, /* d != 128; cols % 32 != 0 on block_axis 1; tile layout with cols != 128 */
+  MXATTN_EALIGN = -3,       /* a pointer is not 16-byte aligned */
+  MXATTN_EWORKSPACE = -4,   /* workspace missing or too small */
+  MXATTN_ECUDA = -5,        /* a CUDA runtime call or the launch failed (see cudaGetLastError) */
+  MXATTN_ETIMEOUT = -6      /* a bounded device-side wait expired (reported by mxattn_device_status) */
+} mxattn_status;
+
+/* Layout of the quantizer's outputs. */
+enum {
+  /* Canonical (for inspection / parity):
+   *   block_axis 1: codes [rows, cols/2] bytes, scales [rows, cols/32] bytes.
+   *   block_axis 0: outputs are TRANSPOSED so that they are contiguous along the block axis, and
+   *                 the block axis is zero-extended to rows_pad = 128*ceil(rows/128):
+   *                 codes [cols, rows_pad/2], scales [cols, rows_pad/32]; a block that is all
+   *                 padding has zero codes and scale byte 127. */
+  MXATTN_LAYOUT_CANONICAL = 0,
+  /* Tile images consumed by the forward kernel (cols must be 128).  Rows are cut into tiles of
+   * 128 (zero-extended); per matrix the outputs are
+   *   codes  [ceil(rows/128)][8192]  and  scales [ceil(rows/128)][512].
+   * Within a tile let (r, c) be (row in tile, block 0..3 along cols) for block_axis 1, and
+   * (column, block of 32 rows 0..3) for block_axis 0; the 16 code bytes of that block sit at
+   *   r*64 + ((c ^ ((r >> 1) & 3)) * 16)        (a 64-byte-swizzled, K-major operand tile)
+   * and its scale byte at  (r % 32)*16 + (r / 32)*4 + c  (the tensor core's scale-factor atom). */
+  MXATTN_LAYOUT_TILE = 1
+};
+
+/* Quantize one bf16 matrix in[rows, cols] to MXFP4 (paper Algorithm 1 for mode UOS; Eq. 5 for
+ * mode OCP; element rounding Eq. 4), canonical layout.
+ *   block_axis 1: blocks run along cols (Q and K: along the head dimension). cols % 32 == 0.
+ *   block_axis 0: blocks run along rows (V: along the token axis), outputs transposed (see above).
+ * codes / e8m0_scales: caller-allocated, sizes as given under MXATTN_LAYOUT_CANONICAL. */
+int mxattn_quantize_mxfp4(const void* in, void* codes, void* e8m0_scales,
+                          int64_t rows, int64_t cols, int block_axis, int mode, void* stream);
+
+/* `batch` independent matrices in[batch][rows, cols] (one per attention head: blocks along the
+ * token axis must not straddle heads), output layout selectable.  Output b starts at
+ * b * (bytes of one matrix's output) in `codes` and `e8m0_scales`. */
+int mxattn_quantize_mxfp4_batched(const void* in, void* codes, void* e8m0_scales, int64_t batch,
+                                  int64_t rows, int64_t cols, int block_axis, int mode, int layout,
+                                  void* stream);
+
+/* Bytes of device scratch the forward pass needs for the quantized Q, K, V tile images, their
+ * scales and a status word.  0 if the shape is unsupported. */
+size_t mxattn_forward_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);
+
+/* Register the scratch used by mxattn_forward.  Caller-owned device memory that must stay valid
+ * until all enqueued forwards have finished.  Process-global: not thread-safe. */
+int mxattn_set_workspace(void* dev_ptr, size_t bytes);
+
+/* MXAttention forward (paper Algorithm 2, lines 3-19; the Hadamard rotation of lines 1-2 is not
+ * part of this call).  q [B,H,Nq,d], k, v [B,H,Nkv,d] bf16; o [B,H,Nq,d] bf16 (fp32 with
+ * MXATTN_FLAG_OUT_FP32).  d must be 128.  Non-causal, no mask.  softmax_scale > 0 multiplies the
+ * quantized product Q-hat K-hat^T (line 9).  KV tiles are 128 keys, visited in ascending order.
+ * Enqueues three quantize launches (Q, K along d; V along tokens) and one fused attention
+ * launch.  Uses the workspace registered with mxattn_set_workspace. */
+int mxattn_forward(const void* q, const void* k, const void* v, void* o,
+                   int B, int H, int64_t Nq, int64_t Nkv, int d,
+                   float softmax_scale, unsigned flags, void* stream);
+
+/* Re-entrant form of mxattn_forward with an explicit workspace. */
+int mxattn_forward_ws(const void* q, const void* k, const void* v, void* o,
+                      int B, int H, int64_t Nq, int64_t Nkv, int d,
+                      float softmax_scale, unsigned flags,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* The fused attention launch alone (Algorithm 2 lines 6-19) on operands already quantized in
+ * MXATTN_LAYOUT_TILE by mxattn_quantize_mxfp4_batched with batch = B*H:
+ * q_* from q (block_axis 1), k_* from k (block_axis 1), v_* from v (block_axis 0).
+ * `status` points to 4 device ints (zeroed by the caller) that receive a non-zero code if a
+ * bounded device-side wait expires. */
+int mxattn_forward_prequantized(const void* q_codes, const void* q_scales,
+                                const void* k_codes, const void* k_scales,
+                                const void* v_codes, const void* v_scales, void* o,
+                                int B, int H, int64_t Nq, int64_t Nkv, int d,
+                                float softmax_scale, unsigned flags, void* status, void* stream);
+
+/* Bytes of device memory mxattn_forward_host needs (inputs, output and workspace). */
+size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags);
+
+/* End-to-end form for callers whose tensors live in HOST memory (pinned memory recommended):
+ * copies q, k, v to the device arena, runs mxattn_forward_ws there, copies o back into o_host and
+ * SYNCHRONIZES `stream` before returning.  `device_arena` is caller-owned device memory of at
+ * least mxattn_forward_host_arena_bytes(). */
+int mxattn_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                        int B, int H, int64_t Nq, int64_t Nkv, int d,
+                        float softmax_scale, unsigned flags,
+                        void* device_arena, size_t arena_bytes, void* stream);
+
+/* Synchronizes `stream`, then copies the workspace's status word to *host_out (host pointer):
+ * 0 = no bounded wait expired since the workspace was last used by a forward. */
+int mxattn_device_status(const void* workspace, int* host_out, void* stream);
+
+/* Number of kernel launches the last forward call of this process enqueued (for accounting). */
+int mxattn_last_launch_count(void);
+
+const char* mxattn_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXATTN_H */

@@ -1,0 +1,172 @@
+// C-ABI entry points that orchestrate the kernels: workspace carving, the three quantize
+// launches plus the fused attention launch (paper Algorithm 2, lines 3-19), and the host-buffer
+// end-to-end form.
+#include "common.cuh"
+
+namespace mxattn {
+
+static int g_launches = 0;
+static void* g_workspace = nullptr;
+static size_t g_workspace_bytes = 0;
+
+void count_launch(int n) { g_launches += n; }
+
+struct WorkspaceLayout {
+  size_t q_codes, q_scales, k_codes, k_scales, v_codes, v_scales, status, total;
+};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool carve(int B, int H, int64_t Nq, int64_t Nkv, int d, WorkspaceLayout* w) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || d != kHeadDim) return false;
+  const size_t bh = (size_t)B * H;
+  const size_t qt = (size_t)((Nq + kTile - 1) / kTile), kt = (size_t)((Nkv + kTile - 1) / kTile);
+  size_t off = 0;
+  w->status = off;   off += 256;
+  w->q_codes = off;  off += align_up(bh * qt * kTileCodeBytes, 256);
+  w->q_scales = off; off += align_up(bh * qt * kTileScaleBytes, 256);
+  w->k_codes = off;  off += align_up(bh * kt * kTileCodeBytes, 256);
+  w->k_scales = off; off += align_up(bh * kt * kTileScaleBytes, 256);
+  w->v_codes = off;  off += align_up(bh * kt * kTileCodeBytes, 256);
+  w->v_scales = off; off += align_up(bh * kt * kTileScaleBytes, 256);
+  w->total = off;
+  return true;
+}
+
+static int forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq,
+                      int64_t Nkv, int d, float softmax_scale, unsigned flags, void* workspace,
+                      size_t workspace_bytes, cudaStream_t stream) {
+  if (!q || !k || !v || !o) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return MXATTN_EALIGN;
+  WorkspaceLayout w;
+  if (!carve(B, H, Nq, Nkv, d, &w)) return MXATTN_EUNSUPPORTED;
+  if (!workspace || workspace_bytes < w.total) return MXATTN_EWORKSPACE;
+  if (!aligned16(workspace)) return MXATTN_EALIGN;
+  g_launches = 0;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const int mode = (flags & MXATTN_FLAG_UOS) ? MXATTN_MODE_UOS : MXATTN_MODE_OCP;
+  const int64_t bh = (int64_t)B * H;
+  if (cudaMemsetAsync(ws + w.status, 0, 16, stream) != cudaSuccess) return MXATTN_ECUDA;
+  int rc;
+  // Algorithm 2 lines 3-5: Q-hat, K-hat (blocks along d), V-hat (blocks along tokens)
+  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  // lines 6-19
+  return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
+                        ws + w.v_scales, o, B, H, Nq, Nkv, softmax_scale, flags,
+                        reinterpret_cast<int*>(ws + w.status), stream);
+}
+
+}  // namespace mxattn
+
+using namespace mxattn;
+
+extern "C" size_t mxattn_forward_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d) {
+  WorkspaceLayout w;
+  return carve(B, H, Nq, Nkv, d, &w) ? w.total : 0;
+}
+
+extern "C" int mxattn_set_workspace(void* dev_ptr, size_t bytes) {
+  if (dev_ptr && !aligned16(dev_ptr)) return MXATTN_EALIGN;
+  g_workspace = dev_ptr;
+  g_workspace_bytes = dev_ptr ? bytes : 0;
+  return MXATTN_OK;
+}
+
+extern "C" int mxattn_forward(const void* q, const void* k, const void* v, void* o, int B, int H,
+                              int64_t Nq, int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                              void* stream) {
+  return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, g_workspace, g_workspace_bytes,
+                    (cudaStream_t)stream);
+}
+
+extern "C" int mxattn_forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H,
+                                 int64_t Nq, int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, workspace_bytes,
+                    (cudaStream_t)stream);
+}
+
+extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_scales, const void* k_codes,
+                                           const void* k_scales, const void* v_codes, const void* v_scales,
+                                           void* o, int B, int H, int64_t Nq, int64_t Nkv, int d,
+                                           float softmax_scale, unsigned flags, void* status, void* stream) {
+  if (!q_codes || !q_scales || !k_codes || !k_scales || !v_codes || !v_scales || !o || !status) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (!aligned16(q_codes) || !aligned16(q_scales) || !aligned16(k_codes) || !aligned16(k_scales) ||
+      !aligned16(v_codes) || !aligned16(v_scales) || !aligned16(o) || !aligned16(status))
+    return MXATTN_EALIGN;
+  g_launches = 0;
+  return launch_forward(q_codes, q_scales, k_codes, k_scales, v_codes, v_scales, o, B, H, Nq, Nkv,
+                        softmax_scale, flags, static_cast<int*>(status), (cudaStream_t)stream);
+}
+
+extern "C" size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags) {
+  WorkspaceLayout w;
+  if (!carve(B, H, Nq, Nkv, d, &w)) return 0;
+  const size_t bh = (size_t)B * H;
+  const size_t qb = align_up(bh * (size_t)Nq * d * 2, 256), kb = align_up(bh * (size_t)Nkv * d * 2, 256);
+  const size_t ob = align_up(bh * (size_t)Nq * d * ((flags & MXATTN_FLAG_OUT_FP32) ? 4 : 2), 256);
+  return qb + 2 * kb + ob + w.total;
+}
+
+extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                                   int B, int H, int64_t Nq, int64_t Nkv, int d, float softmax_scale,
+                                   unsigned flags, void* device_arena, size_t arena_bytes, void* stream_) {
+  if (!q_host || !k_host || !v_host || !o_host) return MXATTN_EINVAL;
+  const size_t need = mxattn_forward_host_arena_bytes(B, H, Nq, Nkv, d, flags);
+  if (need == 0) return (d != kHeadDim) ? MXATTN_EUNSUPPORTED : MXATTN_EINVAL;
+  if (!device_arena || arena_bytes < need) return MXATTN_EWORKSPACE;
+  if (!aligned16(device_arena)) return MXATTN_EALIGN;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const size_t bh = (size_t)B * H;
+  const size_t qn = bh * (size_t)Nq * d * 2, kn = bh * (size_t)Nkv * d * 2;
+  const size_t on = bh * (size_t)Nq * d * ((flags & MXATTN_FLAG_OUT_FP32) ? 4 : 2);
+  uint8_t* a = static_cast<uint8_t*>(device_arena);
+  uint8_t* dq = a;
+  uint8_t* dk = dq + align_up(qn, 256);
+  uint8_t* dv = dk + align_up(kn, 256);
+  uint8_t* dout = dv + align_up(kn, 256);
+  uint8_t* ws = dout + align_up(on, 256);
+  if (cudaMemcpyAsync(dq, q_host, qn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaMemcpyAsync(dk, k_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaMemcpyAsync(dv, v_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
+  const int rc = forward_ws(dq, dk, dv, dout, B, H, Nq, Nkv, d, softmax_scale, flags, ws,
+                            arena_bytes - (size_t)(ws - a), stream);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(o_host, dout, on, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return MXATTN_ECUDA;
+  int st = 0;
+  if (cudaMemcpy(&st, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  return st ? MXATTN_ETIMEOUT : MXATTN_OK;
+}
+
+extern "C" int mxattn_device_status(const void* workspace, int* host_out, void* stream) {
+  if (!workspace || !host_out) return MXATTN_EINVAL;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaMemcpy(host_out, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  return MXATTN_OK;
+}
+
+extern "C" int mxattn_last_launch_count(void) { return g_launches; }
+
+extern "C" const char* mxattn_strerror(int status) {
+  switch (status) {
+    case MXATTN_OK: return "ok";
+    case MXATTN_EINVAL: return "invalid argument";
+    case MXATTN_EUNSUPPORTED: return "unsupported shape";
+    case MXATTN_EALIGN: return "pointer not 16-byte aligned";
+    case MXATTN_EWORKSPACE: return "workspace missing or too small";
+    case MXATTN_ECUDA: return "CUDA runtime error";
+    case MXATTN_ETIMEOUT: return "device-side bounded wait expired";
+    default: return "unknown status";
+  }
+}

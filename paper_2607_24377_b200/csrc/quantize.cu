@@ -1,0 +1,250 @@
+// MXFP4 block quantization kernels (paper Section 2, Eq. 4-7; Algorithm 1) for sm_100a.
+//
+// Both kernels are HBM-bound streaming passes: 2 bytes read, 0.5 + 1/32 bytes written per element.
+//   axis 1 (Q, K): a block is 32 consecutive bf16 of one row.  One thread owns 8 elements (one
+//     128-bit load); the 4 threads of a block combine their maxima with two shuffles.
+//   axis 0 (V): a block is 32 consecutive rows (tokens) of one column.  A CTA stages a
+//     128-token x 128-column slab in shared memory with coalesced 128-bit loads, quantizes down
+//     the columns, and writes the transposed codes through a shared-memory staging tile so that
+//     the global stores stay 128-bit.
+#include "common.cuh"
+
+namespace mxattn {
+
+// ------------------------------------------------------------------------------------------
+// max |x| over the eight bf16 in a uint4, as a bf16 bit pattern (compare as unsigned integers:
+// monotone for non-negative floats).
+__device__ __forceinline__ uint32_t absmax_bf16x8(const uint4& v) {
+  const uint32_t m = 0x7FFF7FFFu;
+  uint32_t a = __vmaxu2(__vmaxu2(v.x & m, v.y & m), __vmaxu2(v.z & m, v.w & m));
+  return max(a & 0xFFFFu, a >> 16);
+}
+
+// Quantize the eight bf16 of `v` with scale 2^-e.
+__device__ __forceinline__ uint32_t quantize_bf16x8(const uint4& v, float inv) {
+  return pack_e2m1x8(bf16lo(v.x) * inv, bf16hi(v.x) * inv, bf16lo(v.y) * inv, bf16hi(v.y) * inv,
+                     bf16lo(v.z) * inv, bf16hi(v.z) * inv, bf16lo(v.w) * inv, bf16hi(v.w) * inv);
+}
+
+constexpr int kQThreads = 256;
+constexpr int kQUnroll = 4;
+
+// ------------------------------------------------------------------------------------------
+// Axis 1.  Work unit = one 16-byte chunk (8 elements).  `n_chunks` counts chunks of the OUTPUT
+// index space: for the canonical layout that is the input itself; for the tile layout rows are
+// padded to a multiple of 128 per matrix and padded rows read as zero.
+template <bool kTileLayout>
+__global__ void __launch_bounds__(kQThreads)
+quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
+                      uint8_t* __restrict__ scales, int64_t n_chunks, int64_t rows,
+                      int64_t rows_pad, bool uos) {
+  const int lane = threadIdx.x & 31;
+  const int64_t stride = (int64_t)gridDim.x * kQThreads;
+  // warp-uniform loop bound: every lane of a warp runs the same number of iterations
+  const int64_t warp_first = (int64_t)blockIdx.x * kQThreads + (threadIdx.x & ~31);
+  for (int64_t base = warp_first; base < n_chunks; base += stride * kQUnroll) {
+    uint4 v[kQUnroll];
+    int64_t idx[kQUnroll];
+#pragma unroll
+    for (int u = 0; u < kQUnroll; ++u) {
+      const int64_t i = base + (int64_t)u * stride + lane;
+      idx[u] = i;
+      v[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (i < n_chunks) {
+        if (kTileLayout) {
+          const int64_t prow = i >> 4;               // padded global row (16 chunks per 128-wide row)
+          const int64_t b = prow / rows_pad;
+          const int64_t rr = prow - b * rows_pad;
+          if (rr < rows) v[u] = __ldg(in + ((b * rows + rr) << 4) + (i & 15));
+        } else {
+          v[u] = __ldg(in + i);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kQUnroll; ++u) {
+      const int64_t i = idx[u];
+      uint32_t m = absmax_bf16x8(v[u]);
+      m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+      m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+      const int e = shared_exponent(m << 16, uos);
+      const uint32_t packed = quantize_bf16x8(v[u], pow2_neg(e));
+      // four consecutive blocks (16 lanes) -> one 32-bit scale word
+      const uint32_t eb = (uint32_t)(e + 127);
+      const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
+      const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
+      const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
+      if (i >= n_chunks) continue;
+      if (kTileLayout) {
+        const int64_t prow = i >> 4;
+        const int64_t tile = prow >> 7;
+        const int r = (int)(prow & 127);
+        const int c = (int)((i >> 2) & 3);
+        codes[(tile * kTileCodeBytes + tile_code_offset(r, c)) / 4 + (i & 3)] = packed;
+        if ((lane & 15) == 0)
+          *reinterpret_cast<uint32_t*>(scales + tile * kTileScaleBytes + tile_scale_offset(r, 0)) =
+              eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
+      } else {
+        codes[i] = packed;
+        if ((lane & 15) == 0) {
+          const int64_t g = i >> 2;                  // block index, multiple of 4 here
+          if (i + 16 <= n_chunks) {
+            *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
+          } else {                                   // ragged end: fewer than 4 blocks left
+            scales[g] = (uint8_t)eb;
+            if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
+            if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
+          }
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Axis 0.  grid = (ceil(cols/128), ceil(rows/128), batch); 256 threads.
+constexpr int kVThreads = 256;
+
+template <bool kTileLayout>
+__global__ void __launch_bounds__(kVThreads)
+quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ codes,
+                      uint8_t* __restrict__ scales, int64_t rows, int64_t cols, int64_t rows_pad,
+                      bool uos) {
+  __shared__ __align__(16) uint16_t s_in[kTile][kTile];           // [token][column] raw bf16
+  __shared__ __align__(16) uint8_t s_codes[kTileCodeBytes];       // [column][64 B] (swizzled if tile layout)
+  __shared__ __align__(16) uint8_t s_scales[kTileScaleBytes];
+
+  const int tid = threadIdx.x;
+  const int64_t col0 = (int64_t)blockIdx.x * kTile;
+  const int64_t row0 = (int64_t)blockIdx.y * kTile;
+  const int64_t b = blockIdx.z;
+  const uint16_t* src = in + b * rows * cols;
+
+  // phase 1: 128 x 128 bf16 slab -> shared, 16 B per thread per step, zero beyond the edges
+#pragma unroll
+  for (int k = 0; k < (kTile * kTile / 8) / kVThreads; ++k) {
+    const int chunk = k * kVThreads + tid;      // 16 chunks per token row
+    const int t = chunk >> 4, cc = (chunk & 15) << 3;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row0 + t < rows && col0 + cc < cols)
+      v = __ldg(reinterpret_cast<const uint4*>(src + (row0 + t) * cols + col0 + cc));
+    *reinterpret_cast<uint4*>(&s_in[t][cc]) = v;
+  }
+  __syncthreads();
+
+  // phase 2: thread -> (column n, token block c); 512 jobs, 2 per thread
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int n = tid & 127;
+    const int c = (tid >> 7) + 2 * k;
+    uint32_t w[16];
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t lo = s_in[c * 32 + 2 * i][n], hi = s_in[c * 32 + 2 * i + 1][n];
+      w[i] = lo | (hi << 16);
+      m = __vmaxu2(m, w[i] & 0x7FFF7FFFu);
+    }
+    m = max(m & 0xFFFFu, m >> 16);
+    const int e = shared_exponent(m << 16, uos);
+    const float inv = pow2_neg(e);
+    uint4 out;
+    out.x = pack_e2m1x8(bf16lo(w[0]) * inv, bf16hi(w[0]) * inv, bf16lo(w[1]) * inv, bf16hi(w[1]) * inv,
+                        bf16lo(w[2]) * inv, bf16hi(w[2]) * inv, bf16lo(w[3]) * inv, bf16hi(w[3]) * inv);
+    out.y = pack_e2m1x8(bf16lo(w[4]) * inv, bf16hi(w[4]) * inv, bf16lo(w[5]) * inv, bf16hi(w[5]) * inv,
+                        bf16lo(w[6]) * inv, bf16hi(w[6]) * inv, bf16lo(w[7]) * inv, bf16hi(w[7]) * inv);
+    out.z = pack_e2m1x8(bf16lo(w[8]) * inv, bf16hi(w[8]) * inv, bf16lo(w[9]) * inv, bf16hi(w[9]) * inv,
+                        bf16lo(w[10]) * inv, bf16hi(w[10]) * inv, bf16lo(w[11]) * inv, bf16hi(w[11]) * inv);
+    out.w = pack_e2m1x8(bf16lo(w[12]) * inv, bf16hi(w[12]) * inv, bf16lo(w[13]) * inv, bf16hi(w[13]) * inv,
+                        bf16lo(w[14]) * inv, bf16hi(w[14]) * inv, bf16lo(w[15]) * inv, bf16hi(w[15]) * inv);
+    const int coff = kTileLayout ? tile_code_offset(n, c) : (n * 64 + c * 16);
+    *reinterpret_cast<uint4*>(&s_codes[coff]) = out;
+    s_scales[kTileLayout ? tile_scale_offset(n, c) : (n * 4 + c)] = (uint8_t)(e + 127);
+  }
+  __syncthreads();
+
+  // phase 3: staged tile -> global
+  if (kTileLayout) {
+    const int64_t tile = b * gridDim.y + blockIdx.y;            // cols == 128: one column tile
+    uint4* dst = reinterpret_cast<uint4*>(codes + tile * kTileCodeBytes);
+#pragma unroll
+    for (int k = 0; k < kTileCodeBytes / 16 / kVThreads; ++k)
+      dst[k * kVThreads + tid] = reinterpret_cast<const uint4*>(s_codes)[k * kVThreads + tid];
+    if (tid < kTileScaleBytes / 16)
+      reinterpret_cast<uint4*>(scales + tile * kTileScaleBytes)[tid] =
+          reinterpret_cast<const uint4*>(s_scales)[tid];
+  } else {
+    // codes [cols, rows_pad/2]: column n owns 64 contiguous bytes of this token tile
+    uint8_t* cdst = codes + b * cols * (rows_pad / 2);
+    uint8_t* sdst = scales + b * cols * (rows_pad / 32);
+#pragma unroll
+    for (int k = 0; k < kTileCodeBytes / 16 / kVThreads; ++k) {
+      const int chunk = k * kVThreads + tid;
+      const int n = chunk >> 2, q = chunk & 3;
+      if (col0 + n < cols)
+        *reinterpret_cast<uint4*>(cdst + (col0 + n) * (rows_pad / 2) + row0 / 2 + q * 16) =
+            reinterpret_cast<const uint4*>(s_codes)[chunk];
+    }
+    if (tid < kTile && col0 + tid < cols)
+      *reinterpret_cast<uint32_t*>(sdst + (col0 + tid) * (rows_pad / 32) + row0 / 32) =
+          reinterpret_cast<const uint32_t*>(s_scales)[tid];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, int64_t rows,
+                    int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream) {
+  if (!in || !codes || !scales) return MXATTN_EINVAL;
+  if (batch <= 0 || rows <= 0 || cols <= 0) return MXATTN_EINVAL;
+  if (block_axis != 0 && block_axis != 1) return MXATTN_EINVAL;
+  if (mode != MXATTN_MODE_OCP && mode != MXATTN_MODE_UOS) return MXATTN_EINVAL;
+  if (layout != MXATTN_LAYOUT_CANONICAL && layout != MXATTN_LAYOUT_TILE) return MXATTN_EINVAL;
+  if (layout == MXATTN_LAYOUT_TILE && cols != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (block_axis == 1 && cols % kBlock != 0) return MXATTN_EUNSUPPORTED;
+  if (block_axis == 0 && cols % 8 != 0) return MXATTN_EUNSUPPORTED;
+  if (!aligned16(in) || !aligned16(codes) || !aligned16(scales)) return MXATTN_EALIGN;
+  const bool uos = (mode == MXATTN_MODE_UOS);
+  const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
+
+  if (block_axis == 1) {
+    const bool tile = (layout == MXATTN_LAYOUT_TILE);
+    const int64_t n_chunks = tile ? batch * rows_pad * 16 : batch * rows * (cols / 8);
+    int64_t blocks = (n_chunks + (int64_t)kQThreads * kQUnroll - 1) / ((int64_t)kQThreads * kQUnroll);
+    const int64_t cap = 148 * 8 * 4;                       // a few waves of resident CTAs
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (tile)
+      quantize_axis1_kernel<true><<<(unsigned)blocks, kQThreads, 0, stream>>>(
+          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rows, rows_pad, uos);
+    else
+      quantize_axis1_kernel<false><<<(unsigned)blocks, kQThreads, 0, stream>>>(
+          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rows, rows_pad, uos);
+  } else {
+    const int64_t ct = (cols + kTile - 1) / kTile, rt = rows_pad / kTile;
+    if (rt > 65535 || batch > 65535) return MXATTN_EUNSUPPORTED;
+    dim3 grid((unsigned)ct, (unsigned)rt, (unsigned)batch);
+    if (layout == MXATTN_LAYOUT_TILE)
+      quantize_axis0_kernel<true><<<grid, kVThreads, 0, stream>>>(
+          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, uos);
+    else
+      quantize_axis0_kernel<false><<<grid, kVThreads, 0, stream>>>(
+          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, uos);
+  }
+  count_launch(1);
+  return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
+}
+
+}  // namespace mxattn
+
+extern "C" int mxattn_quantize_mxfp4(const void* in, void* codes, void* e8m0_scales, int64_t rows,
+                                     int64_t cols, int block_axis, int mode, void* stream) {
+  return mxattn::launch_quantize(in, codes, e8m0_scales, 1, rows, cols, block_axis, mode,
+                                 MXATTN_LAYOUT_CANONICAL, (cudaStream_t)stream);
+}
+
+extern "C" int mxattn_quantize_mxfp4_batched(const void* in, void* codes, void* e8m0_scales,
+                                             int64_t batch, int64_t rows, int64_t cols,
+                                             int block_axis, int mode, int layout, void* stream) {
+  return mxattn::launch_quantize(in, codes, e8m0_scales, batch, rows, cols, block_axis, mode, layout,
+                                 (cudaStream_t)stream);
+}

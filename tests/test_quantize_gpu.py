@@ -1,0 +1,140 @@
+"""Bit-exact parity of the CUDA quantizer with the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from oracle import mxfp4
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+RULE = {0: mxfp4.OCP, 1: mxfp4.UOS}
+
+
+def run_gpu(bits, rows, cols, axis, mode):
+    import paper_2607_24377_b200 as mx
+    x = util.to_dev_bf16(bits)
+    if axis == 1:
+        codes = torch.full((rows, cols // 2), 0xAA, dtype=torch.uint8, device="cuda")
+        scales = torch.full((rows, cols // 32), 0xAA, dtype=torch.uint8, device="cuda")
+    else:
+        rp = -(-rows // 128) * 128
+        codes = torch.full((cols, rp // 2), 0xAA, dtype=torch.uint8, device="cuda")
+        scales = torch.full((cols, rp // 32), 0xAA, dtype=torch.uint8, device="cuda")
+    mx.quantize_mxfp4(x, codes, scales, rows, cols, axis, mode)
+    torch.cuda.synchronize()
+    return codes.cpu().numpy(), scales.cpu().numpy()
+
+
+def gaussian_bits(rows, cols, seed, spread=True):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((rows, cols)).astype(np.float32)
+    if spread:   # vary magnitudes over many binades so every exponent path is hit
+        x *= np.exp2(rng.integers(-12, 12, size=(rows, 1))).astype(np.float32)
+    return si.f32_to_bf16_bits(x)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows,cols", [(1, 32), (3, 32), (7, 96), (1024, 128), (1000, 128), (333, 256), (4099, 128), (65, 4096)])
+def test_axis1_matches_oracle_bit_exact(rows, cols, mode):
+    bits = gaussian_bits(rows, cols, rows * 7 + cols + mode)
+    want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), 1, RULE[mode])
+    got_c, got_s = run_gpu(bits, rows, cols, 1, mode)
+    assert np.array_equal(got_s, want_s)
+    assert np.array_equal(got_c, want_c)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows,cols", [(1, 128), (31, 128), (128, 128), (200, 128), (1024, 128), (1000, 128), (75600 % 4096 + 4096, 128), (300, 64), (260, 264)])
+def test_axis0_matches_oracle_bit_exact(rows, cols, mode):
+    bits = gaussian_bits(rows, cols, rows * 3 + cols + mode)
+    want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), 0, RULE[mode])
+    got_c, got_s = run_gpu(bits, rows, cols, 0, mode)
+    assert np.array_equal(got_s, want_s)
+    assert np.array_equal(got_c, want_c)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_every_bf16_bit_pattern(mode):
+    # all 65536 patterns except Inf/NaN, once alone in a block and once with companions
+    pats = np.array([p for p in range(65536) if (p & 0x7F80) != 0x7F80], dtype=np.uint16)
+    n = pats.size
+    alone = np.zeros((n, 32), np.uint16); alone[:, 5] = pats
+    rng = np.random.default_rng(5)
+    mixed = pats[rng.integers(0, n, size=(4096, 128))]
+    # keep binades close so companions are not all flushed
+    mixed = (mixed & 0x807F) | (np.uint16(0x3F00) + (rng.integers(0, 6, size=mixed.shape).astype(np.uint16) << 7))
+    for bits, cols in ((alone, 32), (mixed, 128)):
+        want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), 1, RULE[mode])
+        got_c, got_s = run_gpu(bits, bits.shape[0], cols, 1, mode)
+        assert np.array_equal(got_s, want_s)
+        assert np.array_equal(got_c, want_c)
+
+
+def test_special_blocks():
+    bits = np.zeros((8, 128), np.uint16)
+    bits[1, :] = 0x8000                               # all -0.0 : zero block, sign kept
+    bits[2, 0] = 0x0001                               # smallest subnormal
+    bits[2, 1] = 0x8040
+    bits[3, 3] = 0x7F7F                               # largest finite
+    bits[3, 4] = 0xFF7F
+    bits[4, :] = si.f32_to_bf16_bits(np.full(128, 7.25, np.float32))      # exact UOS boundary
+    bits[5, :] = si.f32_to_bf16_bits(np.full(128, 7.28125, np.float32))   # one bf16 ulp above
+    bits[6, :32] = si.f32_to_bf16_bits(np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 4.0] * 4, np.float32))  # ties at e = 0
+    bits[7, 64:96] = si.f32_to_bf16_bits(np.linspace(-6, 6, 32).astype(np.float32))
+    for mode in (0, 1):
+        want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), 1, RULE[mode])
+        got_c, got_s = run_gpu(bits, 8, 128, 1, mode)
+        assert np.array_equal(got_s, want_s), mode
+        assert np.array_equal(got_c, want_c), mode
+        want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), 0, RULE[mode])
+        got_c, got_s = run_gpu(bits, 8, 128, 0, mode)
+        assert np.array_equal(got_s, want_s), mode
+        assert np.array_equal(got_c, want_c), mode
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+@pytest.mark.parametrize("rows", [128, 1000, 75600 % 1024 + 1024])
+def test_tile_layout_is_a_permutation_of_the_canonical_one(axis, rows):
+    import paper_2607_24377_b200 as mx
+    batch = 3
+    bits = np.stack([gaussian_bits(rows, 128, 100 + b + rows) for b in range(batch)])
+    x = util.to_dev_bf16(bits)
+    nt = -(-rows // 128)
+    codes = torch.full((batch, nt, 8192), 0xAA, dtype=torch.uint8, device="cuda")
+    scales = torch.full((batch, nt, 512), 0xAA, dtype=torch.uint8, device="cuda")
+    mx.quantize_mxfp4_batched(x, codes, scales, batch, rows, 128, axis, mx.MODE_UOS, mx.LAYOUT_TILE)
+    torch.cuda.synchronize()
+    for b in range(batch):
+        want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits[b]), axis, mxfp4.UOS)
+        tc, ts = (util.canonical_to_tile_axis1 if axis == 1 else util.canonical_to_tile_axis0)(want_c, want_s)
+        assert np.array_equal(scales[b].cpu().numpy(), ts)
+        assert np.array_equal(codes[b].cpu().numpy(), tc)
+
+
+def test_batched_canonical_equals_per_matrix_calls():
+    import paper_2607_24377_b200 as mx
+    batch, rows = 4, 300
+    bits = np.stack([gaussian_bits(rows, 128, 200 + b) for b in range(batch)])
+    x = util.to_dev_bf16(bits)
+    for axis in (0, 1):
+        rp = rows if axis == 1 else 384
+        shape_c = (batch, rows, 64) if axis == 1 else (batch, 128, rp // 2)
+        shape_s = (batch, rows, 4) if axis == 1 else (batch, 128, rp // 32)
+        codes = torch.zeros(shape_c, dtype=torch.uint8, device="cuda")
+        scales = torch.zeros(shape_s, dtype=torch.uint8, device="cuda")
+        mx.quantize_mxfp4_batched(x, codes, scales, batch, rows, 128, axis, mx.MODE_OCP, mx.LAYOUT_CANONICAL)
+        torch.cuda.synchronize()
+        for b in range(batch):
+            want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits[b]), axis, mxfp4.OCP)
+            assert np.array_equal(codes[b].cpu().numpy(), want_c)
+            assert np.array_equal(scales[b].cpu().numpy(), want_s)
+
+
+def test_power_of_two_scaling_shifts_scale_bytes_only():
+    bits = gaussian_bits(512, 128, 9, spread=False)
+    x = si.bf16_bits_to_f32(bits)
+    c0, s0 = run_gpu(bits, 512, 128, 1, 1)
+    c1, s1 = run_gpu(si.f32_to_bf16_bits(x * np.float32(2.0 ** 9)), 512, 128, 1, 1)
+    assert np.array_equal(c0, c1) and np.array_equal(s0.astype(np.int32) + 9, s1.astype(np.int32))
