@@ -1,8 +1,542 @@
-// placeholder, replaced by the fused attention kernel
+// Fused MXFP4 attention forward for sm_100a (paper Algorithm 2, lines 6-19).
+//
+// One CTA owns two query tiles of 128 rows of one head and walks the KV tiles (B_c = 128 keys)
+// in ascending order.  Roles (320 threads):
+//   warps 0-3  softmax group 0 (query tile 0), one thread per query row
+//   warps 4-7  softmax group 1 (query tile 1)
+//   warp  8    producer: bulk async copies (TMA unit) of K-hat / V-hat tile images + scale atoms
+//   warp  9    MMA issuer: block-scaled FP4 tcgen05.mma (kind::mxf4, E8M0 scales), one thread
+//
+// Both GEMMs are dense FP4 contractions with fp32 accumulators in tensor memory:
+//   GEMM 1  S   = Q-hat_t K-hat_j^T              (M=128, N=128, K=128 as two K=64 instructions)
+//   GEMM 2  O_t += P-hat_t [V-hat_j | 1]         (M=128, N=144, K=128)
+// The 16 extra B rows of GEMM 2 hold the constant 1.0, so column 128 of the accumulator is the
+// row sum of the QUANTIZED exponentials, P-hat 1 -- exactly the values the tensor core consumed.
+// That is the PNQ row sum (paper Eq. 22, Algorithm 2 line 14) at no ALU cost; the direct
+// placement (Eq. 12) instead accumulates the unquantized exponentials in a register.
+//
+// Per KV tile a softmax thread (Algorithm 2 lines 10-14, for its row):
+//   reads its 128 scores from tensor memory, takes the four 32-block maxima and the row maximum,
+//   m_new = max(m, rowmax), alpha = exp(m - m_new);  for each block b:
+//     pmax  = exp((bmax_b - m_new) * scale)            -> shared exponent e_b by the UOS / OCP rule
+//     x     = exp2((s - m_new) * scale*log2(e) - e_b)  == P~ / 2^e_b  (the scale folded into the exponent)
+//     codes = RNE-to-E2M1(x), 16 bytes, written into the K-major, 64B-swizzled A-operand tile
+//   and the four scale bytes into the scale-factor atom.  (s - m_new) is formed first so that the
+//   row maximum gives exactly exp(0) = 1, as the paper's Appendix J requires.
+//   If m moved, the thread rescales its accumulator row in tensor memory by alpha (line 15).
+//
+// Tensor-memory map (512 columns): S [0,128) shared by both groups (each group copies its scores
+// to registers at once, so the buffer is free again long before the other group needs it),
+// O_0 [128,272), O_1 [272,416), scale factors from 416.
+//
+// Every wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
 #include "common.cuh"
+
 namespace mxattn {
-int launch_forward(const void*, const void*, const void*, const void*, const void*, const void*, void*,
-                   int, int, int64_t, int64_t, float, unsigned, int*, cudaStream_t) {
-  return MXATTN_EUNSUPPORTED;
+namespace fwd {
+
+constexpr int kThreads = 320;
+constexpr int kStages = 4;
+constexpr int kNV = 144;                         // GEMM 2 N: 128 channels + 16 rows of ones
+constexpr int kVStageBytes = kNV * 64;           // 9216
+
+// shared memory map (byte offsets from a 1024-aligned base)
+constexpr int kOffQ = 0;                                   // 2 x 8192
+constexpr int kOffK = kOffQ + 2 * kTileCodeBytes;          // 4 x 8192
+constexpr int kOffV = kOffK + kStages * kTileCodeBytes;    // 4 x 9216
+constexpr int kOffP = kOffV + kStages * kVStageBytes;      // 2 x 8192
+constexpr int kOffSFQ = kOffP + 2 * kTileCodeBytes;        // 2 x 512
+constexpr int kOffSFK = kOffSFQ + 2 * kTileScaleBytes;     // 4 x 512
+constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
+constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
+constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
+constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
+constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
+constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
+constexpr int kSmemBytes = kOffMisc + 64 + 1024;           // + slack for the 1024 alignment
+
+enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages, BAR_VFULL = BAR_KEMPTY + kStages,
+           BAR_VEMPTY = BAR_VFULL + kStages, BAR_SFULL = BAR_VEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
+           BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2 };
+
+// tensor-memory columns
+constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK = 424,
+                   kColSFV = 432, kColSFP = 448;
+
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
+
+// shared-memory matrix descriptor: K-major, 8-row groups `sbo` bytes apart, swizzle mode `layout`
+// (0 = none, 4 = 64-byte), descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t sbo_bytes, uint32_t layout) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)(layout & 7) << 61);
 }
+
+// instruction descriptor of kind::mxf4.block_scale: A, B = E2M1 (K-major), scales UE8M0, M = 128
+__device__ __forceinline__ uint32_t make_idesc(int n, int ks) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
+         ((uint32_t)(ks * 2) << 29) | ((uint32_t)(ks * 2) << 4);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+               "selp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait was abandoned (own limit reached, or another thread of
+// the CTA already gave up); the caller then skips to the teardown.
+constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at full clock
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status, int code) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (int it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 63) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint32_t saddr) {   // 512-byte scale atom -> 4 columns
+  const uint64_t d = make_desc(saddr, 128, 0);
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+#define TMEM_LD32(taddr, r)                                                                                   \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                      \
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,"  \
+               "%25,%26,%27,%28,%29,%30,%31}, [%32];"                                                         \
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),          \
+                 "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),      \
+                 "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),   \
+                 "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),   \
+                 "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])                                           \
+               : "r"(taddr) : "memory")
+
+#define TMEM_ST32(taddr, r)                                                                                   \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                               \
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,"  \
+               "%25,%26,%27,%28,%29,%30,%31};"                                                                \
+               ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),      \
+                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),\
+                 "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]),          \
+                 "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),          \
+                 "r"(r[30]), "r"(r[31]), "r"(taddr) : "memory")
+
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+struct Params {
+  const uint8_t* q_codes; const uint8_t* q_scales;
+  const uint8_t* k_codes; const uint8_t* k_scales;
+  const uint8_t* v_codes; const uint8_t* v_scales;
+  void* out;
+  int* status;
+  int64_t Nq, Nkv;
+  int q_tiles, kv_tiles, q_pairs;
+  float scale_log2e;    // softmax_scale * log2(e)
+};
+
+// ---------------------------------------------------------------------------------------------
+template <bool kUos, bool kPnq, bool kOutF32>
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + kOffBar;
+  auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.x / p.q_pairs;
+  const int pair = blockIdx.x - bh * p.q_pairs;
+  const int T = p.kv_tiles;
+
+  // ---- setup -------------------------------------------------------------------------------
+  if (tid == 0) {
+    mbar_init(bar(BAR_Q), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(BAR_KFULL + s), 1); mbar_init(bar(BAR_KEMPTY + s), 1);
+      mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
+    }
+    mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
+    mbar_init(bar(BAR_SFREE), 128);
+    mbar_init(bar(BAR_PFULL + 0), 128); mbar_init(bar(BAR_PFULL + 1), 128);
+    mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // constant rows of ones appended to every V stage (E2M1 code 2 = 1.0) and their scale atom (2^0)
+  for (int i = tid; i < kStages * 16 * 64 / 16; i += kThreads) {
+    const int s = i / 64, c = i % 64;
+    reinterpret_cast<uint4*>(smem + kOffV + s * kVStageBytes + kTileCodeBytes)[c] =
+        make_uint4(0x22222222u, 0x22222222u, 0x22222222u, 0x22222222u);
+  }
+  for (int i = tid; i < kTileScaleBytes / 16; i += kThreads)
+    reinterpret_cast<uint4*>(smem + kOffSFOnes)[i] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 8) {
+    // =============================== producer ===============================================
+    if (lane == 0) {
+      const int64_t qt0 = (int64_t)bh * p.q_tiles + 2 * pair;
+      const int64_t qt1 = (2 * pair + 1 < p.q_tiles) ? qt0 + 1 : qt0;     // odd tail: reuse tile 0 (result unused)
+      mbar_expect_tx(bar(BAR_Q), 2 * (kTileCodeBytes + kTileScaleBytes));
+      bulk_g2s(sbase + kOffQ, p.q_codes + qt0 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q));
+      bulk_g2s(sbase + kOffQ + kTileCodeBytes, p.q_codes + qt1 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q));
+      bulk_g2s(sbase + kOffSFQ, p.q_scales + qt0 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q));
+      bulk_g2s(sbase + kOffSFQ + kTileScaleBytes, p.q_scales + qt1 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q));
+      const int64_t kv0 = (int64_t)bh * T;
+      int issued = 0;
+      bool ok = true;
+      for (int j = 0; j < T && ok; ++j) {
+        const int s = j % kStages;
+        const uint32_t ph = (uint32_t)((j / kStages) & 1);
+        if (j >= kStages) ok = mbar_wait(bar(BAR_KEMPTY + s), ph ^ 1u, abort_flag, p.status, 11);
+        if (!ok) break;
+        mbar_expect_tx(bar(BAR_KFULL + s), kTileCodeBytes + kTileScaleBytes);
+        bulk_g2s(sbase + kOffK + s * kTileCodeBytes, p.k_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
+        bulk_g2s(sbase + kOffSFK + s * kTileScaleBytes, p.k_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
+        if (j >= kStages) ok = mbar_wait(bar(BAR_VEMPTY + s), ph ^ 1u, abort_flag, p.status, 12);
+        if (!ok) { issued = j + 1; break; }   // K(j) is in flight, V(j) is not
+        mbar_expect_tx(bar(BAR_VFULL + s), kTileCodeBytes + kTileScaleBytes);
+        bulk_g2s(sbase + kOffV + s * kVStageBytes, p.v_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_VFULL + s));
+        bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_VFULL + s));
+        issued = j + 1;
+      }
+      if (!ok || *abort_flag) {
+        // gave up: let copies already in flight land before the CTA's shared memory is released
+        for (int j = (issued > kStages ? issued - kStages : 0); j < issued; ++j) {
+          const int s = j % kStages;
+          const uint32_t ph = (uint32_t)((j / kStages) & 1);
+          const long long t0 = clock64();
+          while (!mbar_try(bar(BAR_KFULL + s), ph) && clock64() - t0 < 200000000LL) {}
+          while (!mbar_try(bar(BAR_VFULL + s), ph) && clock64() - t0 < 200000000LL) {}
+        }
+        const long long t0 = clock64();
+        while (!mbar_try(bar(BAR_Q), 0) && clock64() - t0 < 200000000LL) {}
+      }
+    }
+  } else if (warp == 9) {
+    // =============================== MMA issuer =============================================
+    if (lane == 0) {
+      bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag, p.status, 21);
+      uint32_t sfree_n = 0;      // completed phases of S_FREE consumed so far
+      auto gemm1 = [&](int t, int j) {      // S = Q_t K_j^T
+        const int s = j % kStages;
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const uint64_t da = make_desc(sbase + kOffQ + t * kTileCodeBytes + ks * 32, 512, 4);
+          const uint64_t db = make_desc(sbase + kOffK + s * kTileCodeBytes + ks * 32, 512, 4);
+          tc_mma(tmem + kColS, da, db, make_idesc(128, ks), tmem + kColSFQ + 4 * t, tmem + kColSFK + 4 * (j & 1), ks);
+        }
+        tc_commit(bar(BAR_SFULL + t));
+      };
+      auto gemm2 = [&](int t, int j) {      // O_t += P_t [V_j | 1]
+        const int s = j % kStages;
+        tc_cp_sf(tmem + kColSFP + 4 * t, sbase + kOffSFP + t * kTileScaleBytes);
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const uint64_t da = make_desc(sbase + kOffP + t * kTileCodeBytes + ks * 32, 512, 4);
+          const uint64_t db = make_desc(sbase + kOffV + s * kVStageBytes + ks * 32, 512, 4);
+          tc_mma(tmem + (t ? kColO1 : kColO0), da, db, make_idesc(kNV, ks), tmem + kColSFP + 4 * t,
+                 tmem + kColSFV + 8 * (j & 1), (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        tc_commit(bar(BAR_ODONE + t));
+      };
+      auto wait_k = [&](int j) {
+        const int s = j % kStages;
+        if (!mbar_wait(bar(BAR_KFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 22)) return false;
+        tc_fence_after();
+        tc_cp_sf(tmem + kColSFK + 4 * (j & 1), sbase + kOffSFK + s * kTileScaleBytes);
+        return true;
+      };
+      auto wait_sfree = [&]() {
+        const bool r = mbar_wait(bar(BAR_SFREE), sfree_n & 1u, abort_flag, p.status, 23);
+        ++sfree_n;
+        tc_fence_after();
+        return r;
+      };
+      if (ok) {
+        tc_fence_after();
+        tc_cp_sf(tmem + kColSFQ + 0, sbase + kOffSFQ);
+        tc_cp_sf(tmem + kColSFQ + 4, sbase + kOffSFQ + kTileScaleBytes);
+        tc_cp_sf(tmem + kColSFV + 4, sbase + kOffSFOnes);        // scales of the ones rows, both slots
+        tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
+      }
+      // prologue: S(0,0), S(1,0), S(0,1)
+      ok = ok && wait_k(0);
+      if (ok) gemm1(0, 0);
+      ok = ok && wait_sfree();
+      if (ok) { gemm1(1, 0); tc_commit(bar(BAR_KEMPTY + 0)); }
+      if (T > 1) {
+        ok = ok && wait_k(1);
+        ok = ok && wait_sfree();
+        if (ok) gemm1(0, 1);
+      }
+      for (int j = 0; j < T && ok; ++j) {
+        const int s = j % kStages;
+        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);
+        ok = ok && mbar_wait(bar(BAR_VFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 25);
+        if (!ok) break;
+        tc_fence_after();
+        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
+        gemm2(0, j);
+        if (j + 1 < T) {
+          ok = wait_sfree();
+          if (!ok) break;
+          gemm1(1, j + 1);
+          tc_commit(bar(BAR_KEMPTY + (j + 1) % kStages));
+        }
+        ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
+        if (!ok) break;
+        tc_fence_after();
+        gemm2(1, j);
+        tc_commit(bar(BAR_VEMPTY + s));
+        if (j + 2 < T) {
+          ok = wait_k(j + 2);
+          ok = ok && wait_sfree();
+          if (!ok) break;
+          gemm1(0, j + 2);
+        }
+      }
+    }
+  } else {
+    // =============================== softmax groups =========================================
+    const int t = warp >> 2;                       // query tile of this group
+    const int row = tid & 127;                     // row within the tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_s = tmem + kColS + lane_addr;
+    const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;
+    const float c = p.scale_log2e;
+    float m_run = -INFINITY;
+    float l_run = 0.0f;                            // direct placement only
+    uint8_t* sP = smem + kOffP + t * kTileCodeBytes;
+    uint8_t* sSFP = smem + kOffSFP + t * kTileScaleBytes;
+    bool ok = true;
+
+    for (int j = 0; j < T; ++j) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t sr[128];
+      TMEM_LD32(t_s + 0, (sr + 0));
+      TMEM_LD32(t_s + 32, (sr + 32));
+      TMEM_LD32(t_s + 64, (sr + 64));
+      TMEM_LD32(t_s + 96, (sr + 96));
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_SFREE));                 // the score buffer may be overwritten
+
+      if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
+        const int valid = (int)(p.Nkv - (int64_t)j * kTile);
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i >= valid) sr[i] = 0xFF800000u;     // -inf
+      }
+      float bmax[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        float mx = __uint_as_float(sr[32 * b]);
+#pragma unroll
+        for (int i = 1; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[32 * b + i]));
+        bmax[b] = mx;
+      }
+      const float m_new = fmaxf(fmaxf(m_run, fmaxf(bmax[0], bmax[1])), fmaxf(bmax[2], bmax[3]));   // line 10
+      const float alpha = ex2((m_run - m_new) * c);                                                // line 11
+      const bool moved = (m_new != m_run) && (j > 0);
+      m_run = m_new;
+
+      if (j > 0) {       // GEMM 2 of the previous tile has read P_t and updated O_t
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), abort_flag, p.status, 32));
+        if (!ok) break;
+        tc_fence_after();
+      }
+      if (__any_sync(0xFFFFFFFFu, moved)) {        // line 15: O~ <- Diag(alpha) O~ (and the PNQ row sum)
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r32[32];
+          TMEM_LD32(t_o + c0, r32);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r32[i] = __float_as_uint(__uint_as_float(r32[i]) * alpha);
+          TMEM_ST32(t_o + c0, r32);
+        }
+        if (kPnq) {                                // column 128: the running row sum P-hat 1
+          uint32_t lr;
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
+          tmem_ld_wait();
+          lr = __float_as_uint(__uint_as_float(lr) * alpha);
+          asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%1], {%0};" ::"r"(lr), "r"(t_o + 128) : "memory");
+        }
+        tmem_st_wait();
+      }
+
+      // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1
+      uint32_t sf_word = 0;
+      float l_tile = 0.0f;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const float pmax = ex2((bmax[b] - m_new) * c);
+        const int e = shared_exponent(__float_as_uint(pmax), kUos);
+        const float ne = (float)(-e);
+        float x[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + i]) - m_new, c, ne));
+        uint4 w;
+        w.x = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+        w.y = pack_e2m1x8(x[8], x[9], x[10], x[11], x[12], x[13], x[14], x[15]);
+        w.z = pack_e2m1x8(x[16], x[17], x[18], x[19], x[20], x[21], x[22], x[23]);
+        w.w = pack_e2m1x8(x[24], x[25], x[26], x[27], x[28], x[29], x[30], x[31]);
+        *reinterpret_cast<uint4*>(sP + tile_code_offset(row, b)) = w;
+        sf_word |= (uint32_t)(e + 127) << (8 * b);
+        if (!kPnq) {                                // Eq. 12: row sum of the UNQUANTIZED exponentials
+          float sx = 0.0f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) sx += x[i];
+          l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);
+        }
+      }
+      *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_word;
+      if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(bar(BAR_PFULL + t));
+    }
+
+    // ---- epilogue: O = O~ / l (line 18) ----
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
+    if (ok) {
+      tc_fence_after();
+      const int qtile = 2 * pair + t;
+      const int64_t grow = (int64_t)qtile * kTile + row;
+      float l = l_run;
+      if (kPnq) {
+        uint32_t lr;
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
+        tmem_ld_wait();
+        l = __uint_as_float(lr);
+      }
+      const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
+      const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim;
+#pragma unroll 1
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r32[32];
+        TMEM_LD32(t_o + c0, r32);
+        tmem_ld_wait();
+        if (store) {
+          if (kOutF32) {
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + obase + c0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(r32[4 * i]) / l, __uint_as_float(r32[4 * i + 1]) / l,
+                                   __uint_as_float(r32[4 * i + 2]) / l, __uint_as_float(r32[4 * i + 3]) / l);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + obase + c0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t h[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float a = __uint_as_float(r32[8 * i + 2 * k]) / l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) / l;
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[k]) : "f"(b2), "f"(a));
+              }
+              dst[i] = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+}  // namespace fwd
+
+int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes, const void* k_scales,
+                   const void* v_codes, const void* v_scales, void* o, int B, int H, int64_t Nq, int64_t Nkv,
+                   float softmax_scale, unsigned flags, int* status, cudaStream_t stream) {
+  using namespace fwd;
+  Params p;
+  p.q_codes = (const uint8_t*)q_codes; p.q_scales = (const uint8_t*)q_scales;
+  p.k_codes = (const uint8_t*)k_codes; p.k_scales = (const uint8_t*)k_scales;
+  p.v_codes = (const uint8_t*)v_codes; p.v_scales = (const uint8_t*)v_scales;
+  p.out = o; p.status = status; p.Nq = Nq; p.Nkv = Nkv;
+  const int64_t qt = (Nq + kTile - 1) / kTile, kt = (Nkv + kTile - 1) / kTile;
+  const int64_t pairs = (qt + 1) / 2;
+  const int64_t grid = (int64_t)B * H * pairs;
+  if (qt > 0x3FFFFFFF || kt > 0x3FFFFFFF || grid > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
+  p.q_tiles = (int)qt; p.kv_tiles = (int)kt; p.q_pairs = (int)pairs;
+  p.scale_log2e = softmax_scale * 1.4426950408889634f;
+
+  const bool uos = flags & MXATTN_FLAG_UOS, pnq = flags & MXATTN_FLAG_PNQ, f32 = flags & MXATTN_FLAG_OUT_FP32;
+  void (*kern)(const Params) = nullptr;
+#define PICK(U, P, F) if (uos == U && pnq == P && f32 == F) kern = attention_kernel<U, P, F>;
+  PICK(false, false, false) PICK(false, false, true) PICK(false, true, false) PICK(false, true, true)
+  PICK(true, false, false) PICK(true, false, true) PICK(true, true, false) PICK(true, true, true)
+#undef PICK
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+    return MXATTN_ECUDA;
+  kern<<<(unsigned)grid, kThreads, kSmemBytes, stream>>>(p);
+  count_launch(1);
+  return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
+}
+
+}  // namespace mxattn

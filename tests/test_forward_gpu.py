@@ -1,0 +1,116 @@
+"""Parity of the fused CUDA attention forward with the oracle (Algorithm 2), through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from oracle import attention
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+REL_L2_TOL = 1e-3      # the tolerance the benchmark spec states for the fp32 output
+MAX_ABS_TOL = 4e-3
+
+
+def run_forward(cfg, q, k, v, uos, pnq, f32=True):
+    import paper_2607_24377_b200 as mx
+    dq, dk, dv = util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v)
+    flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | (mx.FLAG_OUT_FP32 if f32 else 0)
+    out = torch.full((cfg.B, cfg.H, cfg.Nq, cfg.d), float("nan"), dtype=torch.float32 if f32 else torch.bfloat16, device="cuda")
+    ws = torch.empty(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), dtype=torch.uint8, device="cuda")
+    mx.forward_ws(dq, dk, dv, out, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, flags, ws)
+    assert mx.device_status(ws) == 0
+    assert mx.last_launch_count() == 4
+    return out
+
+
+def oracle_out(cfg, q, k, v, uos, pnq):
+    f = util.bits_to_f64
+    return attention.forward(f(q), f(k), f(v), cfg.softmax_scale, uos, pnq)
+
+
+def check(got, want):
+    got = got.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+    mx_abs = np.abs(got - want).max()
+    assert rel <= REL_L2_TOL and mx_abs <= MAX_ABS_TOL, (rel, mx_abs)
+    return rel, mx_abs
+
+
+@pytest.mark.parametrize("uos,pnq", [(True, True), (True, False), (False, False), (False, True)])
+def test_tiny_config_all_variants(uos, pnq):
+    cfg = si.CONFIGS["tiny"]
+    q, k, v = si.make_all(cfg)
+    check(run_forward(cfg, q, k, v, uos, pnq), oracle_out(cfg, q, k, v, uos, pnq))
+
+
+@pytest.mark.parametrize("nq,nkv", [(128, 128), (1, 1), (77, 40), (300, 1000), (256, 200), (640, 1296), (130, 3000)])
+def test_ragged_shapes(nq, nkv):
+    cfg = si.custom_config("r", 1, 3, nq, nkv, 31 + nq + nkv)
+    q, k, v = si.make_all(cfg)
+    check(run_forward(cfg, q, k, v, True, True), oracle_out(cfg, q, k, v, True, True))
+
+
+@pytest.mark.parametrize("recipe", ["outlier", "wan", "hunyuan"])
+def test_structured_inputs_small(recipe):
+    cfg = si.custom_config("s", 2, 2, 384, 1536, 41, recipe)
+    q, k, v = si.make_all(cfg)
+    for uos, pnq in ((True, True), (False, False)):
+        check(run_forward(cfg, q, k, v, uos, pnq), oracle_out(cfg, q, k, v, uos, pnq))
+
+
+def test_bf16_output_is_rounded_fp32_output():
+    cfg = si.custom_config("b", 1, 2, 256, 512, 51)
+    q, k, v = si.make_all(cfg)
+    o32 = run_forward(cfg, q, k, v, True, True, f32=True)
+    o16 = run_forward(cfg, q, k, v, True, True, f32=False)
+    assert torch.equal(o32.to(torch.bfloat16), o16)
+
+
+def test_constant_v_gives_exactly_normalized_rows_under_pnq():
+    # Proposition 1 on the GPU, no oracle involved: V == 1 -> O == 1 under PNQ, != 1 under the direct placement
+    cfg = si.custom_config("c", 1, 2, 256, 1024, 61)
+    q, k, v = si.make_all(cfg)
+    v[:] = si.f32_to_bf16_bits(np.ones(1, np.float32))[0]
+    o = run_forward(cfg, q, k, v, True, True).cpu().numpy()
+    assert np.abs(o - 1.0).max() < 1e-6
+    o = run_forward(cfg, q, k, v, True, False).cpu().numpy()
+    assert np.abs(o - 1.0).max() > 1e-3
+
+
+def test_prequantized_entry_equals_full_forward():
+    import paper_2607_24377_b200 as mx
+    cfg = si.custom_config("p", 1, 2, 300, 700, 71)
+    q, k, v = si.make_all(cfg)
+    full = run_forward(cfg, q, k, v, True, True)
+    bh, qt, kt = cfg.B * cfg.H, -(-cfg.Nq // 128), -(-cfg.Nkv // 128)
+    bufs = []
+    for x, n, nt, axis in ((q, cfg.Nq, qt, 1), (k, cfg.Nkv, kt, 1), (v, cfg.Nkv, kt, 0)):
+        codes = torch.empty((bh, nt, 8192), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((bh, nt, 512), dtype=torch.uint8, device="cuda")
+        mx.quantize_mxfp4_batched(util.to_dev_bf16(x), codes, scales, bh, n, 128, axis, mx.MODE_UOS, mx.LAYOUT_TILE)
+        bufs += [codes, scales]
+    out = torch.zeros((cfg.B, cfg.H, cfg.Nq, 128), dtype=torch.float32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    mx.forward_prequantized(*bufs, out, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, cfg.softmax_scale,
+                            mx.FLAG_UOS | mx.FLAG_PNQ | mx.FLAG_OUT_FP32, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    assert torch.equal(out, full)
+
+
+def test_host_buffer_entry_point():
+    import paper_2607_24377_b200 as mx
+    cfg = si.custom_config("h", 1, 2, 256, 512, 81)
+    q, k, v = si.make_all(cfg)
+    want = run_forward(cfg, q, k, v, True, True).cpu()
+    hq, hk, hv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (q, k, v))
+    ho = torch.empty((cfg.B, cfg.H, cfg.Nq, 128), dtype=torch.float32).pin_memory()
+    flags = mx.FLAG_UOS | mx.FLAG_PNQ | mx.FLAG_OUT_FP32
+    arena = torch.empty(mx.forward_host_arena_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, flags), dtype=torch.uint8, device="cuda")
+    mx.forward_host(hq, hk, hv, ho, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, cfg.softmax_scale, flags, arena)
+    assert torch.equal(ho, want)
