@@ -54,7 +54,8 @@ typedef enum {
   MXATTN_EALIGN = -3,       /* a pointer is not 16-byte aligned */
   MXATTN_EWORKSPACE = -4,   /* workspace missing or too small */
   MXATTN_ECUDA = -5,        /* a CUDA runtime call or the launch failed (see cudaGetLastError) */
-  MXATTN_ETIMEOUT = -6      /* a bounded device-side wait expired (reported by mxattn_device_status) */
+  MXATTN_ETIMEOUT = -6,     /* a bounded device-side wait expired (reported by mxattn_device_status) */
+  MXATTN_ESCRATCH_TOO_SMALL = -7 /* mxattn_forward_static: the problem does not fit the built-in scratch array */
 } mxattn_status;
 
 /* Layout of the quantizer's outputs. */
@@ -137,6 +138,41 @@ int mxattn_forward_host(const void* q_host, const void* k_host, const void* v_ho
                         int B, int H, int64_t Nq, int64_t Nkv, int d,
                         float softmax_scale, unsigned flags,
                         void* device_arena, size_t arena_bytes, void* stream);
+
+/* Size of the scratch array built into the library for mxattn_forward_static (32 MiB). */
+#define MXATTN_STATIC_SCRATCH_BYTES (32u << 20)
+
+/* mxattn_forward for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a host framework whose
+ * device memory is fully pre-planned, in a plugin that must not allocate after start-up, or in a
+ * latency-critical loop that cannot afford an allocator call.  Such a caller can hand over q, k, v
+ * and o (it owns those anyway) but has nowhere to get the forward pass's scratch from, and cannot
+ * call mxattn_set_workspace / mxattn_forward_ws without memory of its own.
+ *
+ * Same arguments, layouts and result as mxattn_forward.  The scratch (the quantized tile images
+ * of Q, K and V, their scales and the status word) is a fixed array of MXATTN_STATIC_SCRATCH_BYTES
+ * in device global memory that is part of the library image: every GPU that loads the library
+ * holds it until the process exits.  The call makes no cudaMalloc / cudaFree and uses no
+ * allocating library routine.
+ *
+ * Limits and rules:
+ *   - mxattn_forward_workspace_bytes(B, H, Nq, Nkv, d) must not exceed
+ *     MXATTN_STATIC_SCRATCH_BYTES, otherwise MXATTN_ESCRATCH_TOO_SMALL is returned and nothing is
+ *     launched (for example B*H = 8 heads of Nq = Nkv = 8192 fit; the Wan2.2-sized problem does not).
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps what the previous call left there.
+ *     Everything the pass relies on being zero (the status word; padding inside the tile images)
+ *     is rewritten by each call.  Two calls whose work overlaps on the GPU (different streams, or
+ *     different host threads) race on the array: serialize them.
+ *   - The status word is the first int of the array; a bounded device-side wait that expires is
+ *     not reported by this entry point itself -- results are then unspecified, as for
+ *     mxattn_forward. */
+int mxattn_forward_static(const void* q, const void* k, const void* v, void* o,
+                          int B, int H, int64_t Nq, int64_t Nkv, int d,
+                          float softmax_scale, unsigned flags, void* stream);
 
 /* Synchronizes `stream`, then copies the workspace's status word to *host_out (host pointer):
  * 0 = no bounded wait expired since the workspace was last used by a forward. */

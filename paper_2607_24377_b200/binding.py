@@ -46,6 +46,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_workspace_bytes.restype = sz
         L.mxattn_set_workspace.argtypes = [vp, sz]
         L.mxattn_forward.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
+        L.mxattn_forward_static.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
         L.mxattn_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
         L.mxattn_forward_prequantized.argtypes = [vp] * 7 + [ci, ci, i64, i64, ci, cf, cu, vp, vp]
         L.mxattn_forward_host_arena_bytes.argtypes = [ci, ci, i64, i64, ci, cu]
@@ -100,6 +101,16 @@ def set_workspace(ws, nbytes=None):
 def forward(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags):
     _check(lib().mxattn_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d,
                                 softmax_scale, flags, _stream()), "mxattn_forward")
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def forward_static(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags):
+    """mxattn_forward_static: the forward pass for callers that may not allocate device memory;
+    its scratch is a fixed 32 MiB array inside the library (see include/mxattn.h for the rules)."""
+    _check(lib().mxattn_forward_static(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d,
+                                       softmax_scale, flags, _stream()), "mxattn_forward_static")
 
 
 def forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):

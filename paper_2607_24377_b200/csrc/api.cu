@@ -149,6 +149,39 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   return st ? MXATTN_ETIMEOUT : MXATTN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Forward pass for callers that cannot allocate device memory.
+//
+// Some hosts of this library may not call cudaMalloc at all: code running inside another
+// framework's memory plan where every byte is pre-assigned, plugins loaded into a process that
+// forbids allocation after start-up, or latency-critical loops where an allocator call (and the
+// implicit synchronization it can bring) is not acceptable.  For them the scratch that
+// mxattn_forward needs lives in the library image itself: a fixed array in device global memory,
+// present on every GPU that loads the library for as long as the process lives.
+static __device__ __align__(256) unsigned char g_static_scratch[MXATTN_STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address, so the
+// address is looked up once per device (with that device current) and cached.
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+extern "C" int mxattn_forward_static(const void* q, const void* k, const void* v, void* o, int B, int H,
+                                     int64_t Nq, int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                                     void* stream) {
+  const size_t need = mxattn_forward_workspace_bytes(B, H, Nq, Nkv, d);
+  if (need == 0) return (d != kHeadDim) ? MXATTN_EUNSUPPORTED : MXATTN_EINVAL;
+  if (need > (size_t)MXATTN_STATIC_SCRATCH_BYTES) return MXATTN_ESCRATCH_TOO_SMALL;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MXATTN_ECUDA;
+  if (!g_static_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return MXATTN_ECUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, g_static_scratch_ptr[dev],
+                    (size_t)MXATTN_STATIC_SCRATCH_BYTES, (cudaStream_t)stream);
+}
+
 extern "C" int mxattn_device_status(const void* workspace, int* host_out, void* stream) {
   if (!workspace || !host_out) return MXATTN_EINVAL;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MXATTN_ECUDA;
@@ -167,6 +200,9 @@ extern "C" const char* mxattn_strerror(int status) {
     case MXATTN_EWORKSPACE: return "workspace missing or too small";
     case MXATTN_ECUDA: return "CUDA runtime error";
     case MXATTN_ETIMEOUT: return "device-side bounded wait expired";
+    case MXATTN_ESCRATCH_TOO_SMALL:
+      return "problem needs more scratch than the built-in static array holds (MXATTN_STATIC_SCRATCH_BYTES); "
+             "use mxattn_forward_ws with caller-provided memory";
     default: return "unknown status";
   }
 }
