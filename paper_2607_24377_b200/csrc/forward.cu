@@ -1,11 +1,13 @@
 // Fused MXFP4 attention forward for sm_100a (paper Algorithm 2, lines 6-19).
 //
 // One CTA owns two query tiles of 128 rows of one head and walks the KV tiles (B_c = 128 keys)
-// in ascending order.  Roles (320 threads):
-//   warps 0-3  softmax group 0 (query tile 0), one thread per query row
-//   warps 4-7  softmax group 1 (query tile 1)
-//   warp  8    producer: bulk async copies (TMA unit) of K-hat / V-hat tile images + scale atoms
-//   warp  9    MMA issuer: block-scaled FP4 tcgen05.mma (kind::mxf4, E8M0 scales), one thread
+// in ascending order.  Roles (576 threads):
+//   warps 0-7   softmax group 0 (query tile 0): two threads per query row, 64 key columns each
+//               (warps 0-3 take columns 0-63, warps 4-7 columns 64-127; warp w works on the
+//               tensor-memory lanes 32*(w%4) .. +31, i.e. rows 32*(w%4) .. +31 of the tile)
+//   warps 8-15  softmax group 1 (query tile 1), same split
+//   warp  16    producer: bulk async copies (TMA unit) of K-hat / V-hat tile images + scale atoms
+//   warp  17    MMA issuer: block-scaled FP4 tcgen05.mma (kind::mxf4, E8M0 scales), one thread
 //
 // Both GEMMs are dense FP4 contractions with fp32 accumulators in tensor memory:
 //   GEMM 1  S   = Q-hat_t K-hat_j^T              (M=128, N=128, K=128 as two K=64 instructions)
@@ -15,15 +17,19 @@
 // That is the PNQ row sum (paper Eq. 22, Algorithm 2 line 14) at no ALU cost; the direct
 // placement (Eq. 12) instead accumulates the unquantized exponentials in a register.
 //
-// Per KV tile a softmax thread (Algorithm 2 lines 10-14, for its row):
-//   reads its 128 scores from tensor memory, takes the four 32-block maxima and the row maximum,
-//   m_new = max(m, rowmax), alpha = exp(m - m_new);  for each block b:
-//     pmax  = exp((bmax_b - m_new) * scale)            -> shared exponent e_b by the UOS / OCP rule
-//     x     = exp2((s - m_new) * scale*log2(e) - e_b)  == P~ / 2^e_b  (the scale folded into the exponent)
+// Per KV tile a softmax thread (Algorithm 2 lines 10-14, for its half row):
+//   reads its 64 scores from tensor memory, takes its two 32-block maxima, exchanges the half-row
+//   maximum with its partner thread through shared memory, m_new = max(m, rowmax),
+//   alpha = exp(m - m_new);  for each of its blocks b:
+//     pmax  = exp2((bmax_b - m_new) * c)        -> shared exponent e_b by the UOS / OCP rule
+//     x     = exp2(s * c - (m_new * c + e_b))   == P~ / 2^e_b   (the block scale folded into the exponent)
 //     codes = RNE-to-E2M1(x), 16 bytes, written into the K-major, 64B-swizzled A-operand tile
-//   and the four scale bytes into the scale-factor atom.  (s - m_new) is formed first so that the
-//   row maximum gives exactly exp(0) = 1, as the paper's Appendix J requires.
-//   If m moved, the thread rescales its accumulator row in tensor memory by alpha (line 15).
+//   and its two scale bytes into the scale-factor atom (c = softmax_scale * log2 e).  The
+//   difference (bmax_b - m_new) is formed exactly first, so the block holding the row maximum sees
+//   pmax = exp2(0) = 1 exactly and gets the scale the paper's Appendix J derives; the elements
+//   themselves take one fused multiply-add each.
+//   If m moved, the thread rescales its 64 accumulator columns in tensor memory by alpha
+//   (line 15); those tensor-memory round trips are interleaved with the exponentials.
 //
 // Tensor-memory map (512 columns): S [0,128) shared by both groups (each group copies its scores
 // to registers at once, so the buffer is free again long before the other group needs it),
@@ -35,7 +41,8 @@
 namespace mxattn {
 namespace fwd {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 576;                   // 16 softmax warps + producer + MMA issuer
+constexpr int kSoftmaxWarps = 16;
 constexpr int kStages = 4;
 constexpr int kNV = 144;                         // GEMM 2 N: 128 channels + 16 rows of ones
 constexpr int kVStageBytes = kNV * 64;           // 9216
@@ -53,7 +60,8 @@ constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
 constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
-constexpr int kSmemBytes = kOffMisc + 64 + 1024;           // + slack for the 1024 alignment
+constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
+constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
 
 enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages, BAR_VFULL = BAR_KEMPTY + kStages,
            BAR_VEMPTY = BAR_VFULL + kStages, BAR_SFULL = BAR_VEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
@@ -66,6 +74,11 @@ constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -164,6 +177,23 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
                  "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),          \
                  "r"(r[30]), "r"(r[31]), "r"(taddr) : "memory")
 
+#define TMEM_LD8(taddr, r)                                                                            \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"              \
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) \
+               : "r"(taddr) : "memory")
+#define TMEM_ST8(taddr, r)                                                                            \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"              \
+               ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(taddr) : "memory")
+#define TMEM_LD16(taddr, r)                                                                                   \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),    \
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) \
+               : "r"(taddr) : "memory")
+#define TMEM_ST16(taddr, r)                                                                                   \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};" \
+               ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),  \
+                 "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr) : "memory")
+
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -190,6 +220,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (*reinterpret_cast<volatile int*>(p.status) != 0) return;   // an earlier CTA gave up: drain the grid quickly
   const int bh = blockIdx.x / p.q_pairs;
   const int pair = blockIdx.x - bh * p.q_pairs;
   const int T = p.kv_tiles;
@@ -202,8 +233,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
     }
     mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-    mbar_init(bar(BAR_SFREE), 128);
-    mbar_init(bar(BAR_PFULL + 0), 128); mbar_init(bar(BAR_PFULL + 1), 128);
+    mbar_init(bar(BAR_SFREE), 256);
+    mbar_init(bar(BAR_PFULL + 0), 256); mbar_init(bar(BAR_PFULL + 1), 256);
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -217,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   for (int i = tid; i < kTileScaleBytes / 16; i += kThreads)
     reinterpret_cast<uint4*>(smem + kOffSFOnes)[i] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  if (warp == 9) {
+  if (warp == kSoftmaxWarps + 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -226,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == kSoftmaxWarps) {
     // =============================== producer ===============================================
     if (lane == 0) {
       const int64_t qt0 = (int64_t)bh * p.q_tiles + 2 * pair;
@@ -267,7 +298,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         while (!mbar_try(bar(BAR_Q), 0) && clock64() - t0 < 200000000LL) {}
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kSoftmaxWarps + 1) {
     // =============================== MMA issuer =============================================
     if (lane == 0) {
       bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag, p.status, 21);
@@ -351,68 +382,98 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       }
     }
-  } else {
+  } else if (warp < kSoftmaxWarps) {
     // =============================== softmax groups =========================================
-    const int t = warp >> 2;                       // query tile of this group
-    const int row = tid & 127;                     // row within the tile == TMEM lane
+    const int t = warp >> 3;                       // query tile of this group
+    const int h = (warp >> 2) & 1;                 // which 64 key columns of the tile
+    const int row = (warp & 3) * 32 + lane;        // row within the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_s = tmem + kColS + lane_addr;
-    const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;
+    const uint32_t t_s = tmem + kColS + lane_addr + 64 * h;
+    const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;     // column 0 of this row's accumulator
     const float c = p.scale_log2e;
     float m_run = -INFINITY;
-    float l_run = 0.0f;                            // direct placement only
+    float l_run = 0.0f;                            // direct placement only (this thread's 64 columns)
     uint8_t* sP = smem + kOffP + t * kTileCodeBytes;
     uint8_t* sSFP = smem + kOffSFP + t * kTileScaleBytes;
+    float* sMax = reinterpret_cast<float*>(smem + kOffMax);
     bool ok = true;
 
     for (int j = 0; j < T; ++j) {
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
       if (!ok) break;
       tc_fence_after();
-      uint32_t sr[128];
+      uint32_t sr[64];
       TMEM_LD32(t_s + 0, (sr + 0));
       TMEM_LD32(t_s + 32, (sr + 32));
-      TMEM_LD32(t_s + 64, (sr + 64));
-      TMEM_LD32(t_s + 96, (sr + 96));
       tmem_ld_wait();
       tc_fence_before();
       mbar_arrive(bar(BAR_SFREE));                 // the score buffer may be overwritten
 
       if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
-        const int valid = (int)(p.Nkv - (int64_t)j * kTile);
+        const int valid = (int)(p.Nkv - (int64_t)j * kTile) - 64 * h;
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < 64; ++i)
           if (i >= valid) sr[i] = 0xFF800000u;     // -inf
       }
-      float bmax[4];
+      float bmax[2];
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        float mx = __uint_as_float(sr[32 * b]);
+      for (int b = 0; b < 2; ++b) {
+        float mx = max3(__uint_as_float(sr[32 * b]), __uint_as_float(sr[32 * b + 1]), __uint_as_float(sr[32 * b + 2]));
 #pragma unroll
-        for (int i = 1; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[32 * b + i]));
-        bmax[b] = mx;
+        for (int i = 3; i < 31; i += 2) mx = max3(mx, __uint_as_float(sr[32 * b + i]), __uint_as_float(sr[32 * b + i + 1]));
+        bmax[b] = fmaxf(mx, __uint_as_float(sr[32 * b + 31]));
       }
-      const float m_new = fmaxf(fmaxf(m_run, fmaxf(bmax[0], bmax[1])), fmaxf(bmax[2], bmax[3]));   // line 10
-      const float alpha = ex2((m_run - m_new) * c);                                                // line 11
+      // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
+      float* mslot = sMax + ((j & 1) * 2 + t) * 256;
+      mslot[h * 128 + row] = fmaxf(bmax[0], bmax[1]);
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+      const float m_new = max3(m_run, fmaxf(bmax[0], bmax[1]), mslot[(h ^ 1) * 128 + row]);        // line 10
+      const float alpha = ex2((m_run - m_new) * c);                                                 // line 11
       const bool moved = (m_new != m_run) && (j > 0);
       m_run = m_new;
+      const float nmc = -(m_new * c);
 
       if (j > 0) {       // GEMM 2 of the previous tile has read P_t and updated O_t
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), abort_flag, p.status, 32));
         if (!ok) break;
         tc_fence_after();
       }
-      if (__any_sync(0xFFFFFFFFu, moved)) {        // line 15: O~ <- Diag(alpha) O~ (and the PNQ row sum)
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r32[32];
-          TMEM_LD32(t_o + c0, r32);
-          tmem_ld_wait();
+      const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
+
+      // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1
+      uint32_t sf_half = 0;
+      float l_tile = 0.0f;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) r32[i] = __float_as_uint(__uint_as_float(r32[i]) * alpha);
-          TMEM_ST32(t_o + c0, r32);
+      for (int b = 0; b < 2; ++b) {
+        const float pmax = ex2((bmax[b] - m_new) * c);
+        const int e = shared_exponent(__float_as_uint(pmax), kUos);
+        const float nb = nmc - (float)e;
+        uint4 w;
+        float sx = 0.0f;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {               // 8 elements per step, with 8 accumulator columns in flight
+          uint32_t oc[8];
+          const uint32_t t_oc = t_o + 64 * h + 32 * b + 8 * g;
+          if (rescale) TMEM_LD8(t_oc, oc);
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + 8 * g + i]), c, nb));
+          const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+          if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
+          if (!kPnq) sx += ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
+          if (rescale) {
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) oc[i] = __float_as_uint(__uint_as_float(oc[i]) * alpha);
+            TMEM_ST8(t_oc, oc);
+          }
         }
-        if (kPnq) {                                // column 128: the running row sum P-hat 1
+        *reinterpret_cast<uint4*>(sP + tile_code_offset(row, 2 * h + b)) = w;
+        sf_half |= (uint32_t)(e + 127) << (8 * b);
+        if (!kPnq) l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);   // Eq. 12
+      }
+      if (rescale) {
+        if (kPnq && h == 0) {                      // column 128: the running row sum P-hat 1
           uint32_t lr;
           asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
           tmem_ld_wait();
@@ -421,33 +482,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
         tmem_st_wait();
       }
-
-      // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1
-      uint32_t sf_word = 0;
-      float l_tile = 0.0f;
-#pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const float pmax = ex2((bmax[b] - m_new) * c);
-        const int e = shared_exponent(__float_as_uint(pmax), kUos);
-        const float ne = (float)(-e);
-        float x[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + i]) - m_new, c, ne));
-        uint4 w;
-        w.x = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
-        w.y = pack_e2m1x8(x[8], x[9], x[10], x[11], x[12], x[13], x[14], x[15]);
-        w.z = pack_e2m1x8(x[16], x[17], x[18], x[19], x[20], x[21], x[22], x[23]);
-        w.w = pack_e2m1x8(x[24], x[25], x[26], x[27], x[28], x[29], x[30], x[31]);
-        *reinterpret_cast<uint4*>(sP + tile_code_offset(row, b)) = w;
-        sf_word |= (uint32_t)(e + 127) << (8 * b);
-        if (!kPnq) {                                // Eq. 12: row sum of the UNQUANTIZED exponentials
-          float sx = 0.0f;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) sx += x[i];
-          l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);
-        }
-      }
-      *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_word;
+      *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
@@ -456,11 +491,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
 
     // ---- epilogue: O = O~ / l (line 18) ----
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
+    float l = l_run;
+    if (!kPnq) {                                   // add the partner's half of the row sum
+      float* mslot = sMax + ((T & 1) * 2 + t) * 256;
+      mslot[h * 128 + row] = l_run;
+      asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+      l = l_run + mslot[(h ^ 1) * 128 + row];
+    }
     if (ok) {
       tc_fence_after();
       const int qtile = 2 * pair + t;
       const int64_t grow = (int64_t)qtile * kTile + row;
-      float l = l_run;
       if (kPnq) {
         uint32_t lr;
         asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
@@ -468,11 +509,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         l = __uint_as_float(lr);
       }
       const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
-      const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim;
+      const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + 64 * h;
 #pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
+      for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t r32[32];
-        TMEM_LD32(t_o + c0, r32);
+        TMEM_LD32(t_o + 64 * h + c0, r32);
         tmem_ld_wait();
         if (store) {
           if (kOutF32) {
@@ -485,13 +526,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
             uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + obase + c0);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              uint32_t h[4];
+              uint32_t hh[4];
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
                 const float a = __uint_as_float(r32[8 * i + 2 * k]) / l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) / l;
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[k]) : "f"(b2), "f"(a));
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hh[k]) : "f"(b2), "f"(a));
               }
-              dst[i] = make_uint4(h[0], h[1], h[2], h[3]);
+              dst[i] = make_uint4(hh[0], hh[1], hh[2], hh[3]);
             }
           }
         }
@@ -502,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   // ---- teardown ------------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kSoftmaxWarps + 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
   }
