@@ -36,6 +36,8 @@
 // O_0 [128,272), O_1 [272,416), scale factors from 416.
 //
 // Every wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace mxattn {
@@ -58,7 +60,7 @@ constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
 constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
 constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
-constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
+constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2 + 1;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
 constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
@@ -109,9 +111,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+  // the third operand is a suspend-time hint (ns): the thread sleeps in hardware instead of spinning
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
                "selp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+               : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return ok != 0;
 }
 
@@ -123,8 +126,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
+#ifdef EXP_TIMELINE
+    if (code >= 31 && blockIdx.x == 300 && (threadIdx.x == 0 || threadIdx.x == 256)) atomicAdd(status + 8 + (code - 31) + 4 * (threadIdx.x >> 8), 1);
+    if (code < 31 && blockIdx.x == 300) atomicAdd(status + 4000 + code, 1);
+#endif
     if (mbar_try(bar, parity)) return true;
-    if ((it & 63) == 0) {
+    if ((it & 15) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
@@ -233,8 +240,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
     }
     mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-    mbar_init(bar(BAR_SFREE), 256);
-    mbar_init(bar(BAR_PFULL + 0), 256); mbar_init(bar(BAR_PFULL + 1), 256);
+    mbar_init(bar(BAR_SFREE), 8);
+    mbar_init(bar(kNumBars - 1), 8);
+    mbar_init(bar(BAR_PFULL + 0), 8); mbar_init(bar(BAR_PFULL + 1), 8);   // one arrival per softmax warp
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -345,6 +353,47 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         tc_cp_sf(tmem + kColSFV + 4, sbase + kOffSFOnes);        // scales of the ones rows, both slots
         tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
       }
+#ifdef EXP_TWO_S
+      auto gemm1x = [&](int t, int j) {
+        const int s = j % kStages;
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const uint64_t da = make_desc(sbase + kOffQ + t * kTileCodeBytes + ks * 32, 512, 4);
+          const uint64_t db = make_desc(sbase + kOffK + s * kTileCodeBytes + ks * 32, 512, 4);
+          tc_mma(tmem + kColS + 128 * t, da, db, make_idesc(128, ks), tmem + kColSFQ + 4 * t, tmem + kColSFK + 4 * (j & 1), ks);
+        }
+        tc_commit(bar(BAR_SFULL + t));
+      };
+      ok = ok && wait_k(0);
+      if (ok) { gemm1x(0, 0); gemm1x(1, 0); tc_commit(bar(BAR_KEMPTY + 0)); }
+      for (int j = 0; j < T && ok; ++j) {
+        const int s = j % kStages;
+        if (j + 1 < T) {
+          ok = wait_k(j + 1);
+          ok = ok && mbar_wait(bar(BAR_SFREE), (uint32_t)(j & 1), abort_flag, p.status, 23);
+          if (!ok) break;
+          tc_fence_after();
+          gemm1x(0, j + 1);
+          ok = mbar_wait(bar(kNumBars - 1), (uint32_t)(j & 1), abort_flag, p.status, 23);
+          if (!ok) break;
+          tc_fence_after();
+          gemm1x(1, j + 1);
+          tc_commit(bar(BAR_KEMPTY + (j + 1) % kStages));
+        }
+        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);
+        ok = ok && mbar_wait(bar(BAR_VFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 25);
+        if (!ok) break;
+        tc_fence_after();
+        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
+        gemm2(0, j);
+        ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
+        if (!ok) break;
+        tc_fence_after();
+        gemm2(1, j);
+        tc_commit(bar(BAR_VEMPTY + s));
+      }
+    }
+#else
       // prologue: S(0,0), S(1,0), S(0,1)
       ok = ok && wait_k(0);
       if (ok) gemm1(0, 0);
@@ -382,13 +431,18 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       }
     }
+#endif
   } else if (warp < kSoftmaxWarps) {
     // =============================== softmax groups =========================================
     const int t = warp >> 3;                       // query tile of this group
     const int h = (warp >> 2) & 1;                 // which 64 key columns of the tile
     const int row = (warp & 3) * 32 + lane;        // row within the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+#ifdef EXP_TWO_S
+    const uint32_t t_s = tmem + kColS + 128 * t + lane_addr + 64 * h;
+#else
     const uint32_t t_s = tmem + kColS + lane_addr + 64 * h;
+#endif
     const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;     // column 0 of this row's accumulator
     const float c = p.scale_log2e;
     float m_run = -INFINITY;
@@ -396,18 +450,33 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     uint8_t* sP = smem + kOffP + t * kTileCodeBytes;
     uint8_t* sSFP = smem + kOffSFP + t * kTileScaleBytes;
     float* sMax = reinterpret_cast<float*>(smem + kOffMax);
+    const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
     bool ok = true;
 
+#ifdef EXP_TIMELINE
+#define TL(k) if (blockIdx.x == 300 && lane == 0 && (warp == 0 || warp == 8 || warp == 4) && j >= 40 && j < 48) \
+    reinterpret_cast<long long*>(p.status + 16)[((warp >> 2) * 8 + (j - 40)) * 8 + (k)] = clock64();
+#else
+#define TL(k)
+#endif
     for (int j = 0; j < T; ++j) {
+      TL(0)
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
       TMEM_LD32(t_s + 0, (sr + 0));
       TMEM_LD32(t_s + 32, (sr + 32));
+      TL(1)
       tmem_ld_wait();
+      TL(2)
       tc_fence_before();
-      mbar_arrive(bar(BAR_SFREE));                 // the score buffer may be overwritten
+      __syncwarp();
+#ifdef EXP_TWO_S
+      if (lane == 0) mbar_arrive(bar(t ? kNumBars - 1 : BAR_SFREE));
+#else
+      if (lane == 0) mbar_arrive(bar(BAR_SFREE));  // the score buffer may be overwritten
+#endif
 
       if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
         const int valid = (int)(p.Nkv - (int64_t)j * kTile) - 64 * h;
@@ -417,16 +486,24 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       }
       float bmax[2];
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {
-        float mx = max3(__uint_as_float(sr[32 * b]), __uint_as_float(sr[32 * b + 1]), __uint_as_float(sr[32 * b + 2]));
+      for (int b = 0; b < 2; ++b) {                 // four independent chains of 8, then combine
+        float q4[4];
 #pragma unroll
-        for (int i = 3; i < 31; i += 2) mx = max3(mx, __uint_as_float(sr[32 * b + i]), __uint_as_float(sr[32 * b + i + 1]));
-        bmax[b] = fmaxf(mx, __uint_as_float(sr[32 * b + 31]));
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t* v = sr + 32 * b + 8 * u;
+          float mx = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+          mx = max3(mx, __uint_as_float(v[3]), __uint_as_float(v[4]));
+          mx = max3(mx, __uint_as_float(v[5]), __uint_as_float(v[6]));
+          q4[u] = fmaxf(mx, __uint_as_float(v[7]));
+        }
+        bmax[b] = fmaxf(max3(q4[0], q4[1], q4[2]), q4[3]);
       }
       // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
       float* mslot = sMax + ((j & 1) * 2 + t) * 256;
       mslot[h * 128 + row] = fmaxf(bmax[0], bmax[1]);
-      asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+      TL(3)
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
+      TL(4)
       const float m_new = max3(m_run, fmaxf(bmax[0], bmax[1]), mslot[(h ^ 1) * 128 + row]);        // line 10
       const float alpha = ex2((m_run - m_new) * c);                                                 // line 11
       const bool moved = (m_new != m_run) && (j > 0);
@@ -438,55 +515,65 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         if (!ok) break;
         tc_fence_after();
       }
+      TL(5)
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
 
-      // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1
+      // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1.  Two
+      // straight-line versions: the common one, and one that also rescales this thread's 64
+      // accumulator columns with the tensor-memory round trips interleaved into the exponentials.
       uint32_t sf_half = 0;
       float l_tile = 0.0f;
+      auto tile_body = [&](auto resc_tag) {
+        constexpr bool kResc = decltype(resc_tag)::value;
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {
-        const float pmax = ex2((bmax[b] - m_new) * c);
-        const int e = shared_exponent(__float_as_uint(pmax), kUos);
-        const float nb = nmc - (float)e;
-        uint4 w;
-        float sx = 0.0f;
+        for (int b = 0; b < 2; ++b) {
+          const float pmax = ex2((bmax[b] - m_new) * c);
+          const int e = shared_exponent(__float_as_uint(pmax), kUos);
+          const float nb = nmc - (float)e;
+          uint4 w;
+          float sx = 0.0f;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {               // 8 elements per step, with 8 accumulator columns in flight
-          uint32_t oc[8];
-          const uint32_t t_oc = t_o + 64 * h + 32 * b + 8 * g;
-          if (rescale) TMEM_LD8(t_oc, oc);
-          float x[8];
+          for (int g = 0; g < 4; ++g) {             // 8 elements per step (8 accumulator columns in flight)
+            uint32_t oc[8];
+            const uint32_t t_oc = t_o + 64 * h + 32 * b + 8 * g;
+            if (kResc) TMEM_LD8(t_oc, oc);
+            float x[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + 8 * g + i]), c, nb));
-          const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
-          if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
-          if (!kPnq) sx += ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
-          if (rescale) {
-            tmem_ld_wait();
+            for (int i = 0; i < 8; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + 8 * g + i]), c, nb));
+            const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+            if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
+            if (!kPnq) sx += ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
+            if (kResc) {
+              tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 8; ++i) oc[i] = __float_as_uint(__uint_as_float(oc[i]) * alpha);
-            TMEM_ST8(t_oc, oc);
+              for (int i = 0; i < 8; ++i) oc[i] = __float_as_uint(__uint_as_float(oc[i]) * alpha);
+              TMEM_ST8(t_oc, oc);
+            }
           }
+          *reinterpret_cast<uint4*>(sP + tile_code_offset(row, 2 * h + b)) = w;
+          sf_half |= (uint32_t)(e + 127) << (8 * b);
+          if (!kPnq) l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);   // Eq. 12
         }
-        *reinterpret_cast<uint4*>(sP + tile_code_offset(row, 2 * h + b)) = w;
-        sf_half |= (uint32_t)(e + 127) << (8 * b);
-        if (!kPnq) l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);   // Eq. 12
-      }
-      if (rescale) {
-        if (kPnq && h == 0) {                      // column 128: the running row sum P-hat 1
-          uint32_t lr;
-          asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
-          tmem_ld_wait();
-          lr = __float_as_uint(__uint_as_float(lr) * alpha);
-          asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%1], {%0};" ::"r"(lr), "r"(t_o + 128) : "memory");
+        if (kResc) {
+          if (kPnq && h == 0) {                     // column 128: the running row sum P-hat 1
+            uint32_t lr;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
+            tmem_ld_wait();
+            lr = __float_as_uint(__uint_as_float(lr) * alpha);
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%1], {%0};" ::"r"(lr), "r"(t_o + 128) : "memory");
+          }
+          tmem_st_wait();
         }
-        tmem_st_wait();
-      }
+      };
+      if (rescale) tile_body(std::true_type{}); else tile_body(std::false_type{});
+      TL(6)
       *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
-      mbar_arrive(bar(BAR_PFULL + t));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
+      TL(7)
     }
 
     // ---- epilogue: O = O~ / l (line 18) ----
@@ -495,7 +582,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     if (!kPnq) {                                   // add the partner's half of the row sum
       float* mslot = sMax + ((T & 1) * 2 + t) * 256;
       mslot[h * 128 + row] = l_run;
-      asm volatile("bar.sync %0, 256;" ::"r"(1 + t) : "memory");
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       l = l_run + mslot[(h ^ 1) * 128 + row];
     }
     if (ok) {
