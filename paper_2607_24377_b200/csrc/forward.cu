@@ -118,6 +118,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {     // non-blocking
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+               "selp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false if the wait was abandoned (own limit reached, or another thread of
 // the CTA already gave up); the caller then skips to the teardown.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at full clock
@@ -501,22 +509,27 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
       float* mslot = sMax + ((j & 1) * 2 + t) * 256;
       mslot[h * 128 + row] = fmaxf(bmax[0], bmax[1]);
+      // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t
+      // or rescales O_t; probe that barrier now so its latency overlaps the pair barrier
+      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
       TL(3)
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
       TL(4)
       const float m_new = max3(m_run, fmaxf(bmax[0], bmax[1]), mslot[(h ^ 1) * 128 + row]);        // line 10
-      const float alpha = ex2((m_run - m_new) * c);                                                 // line 11
       const bool moved = (m_new != m_run) && (j > 0);
+      const float m_old = m_run;
       m_run = m_new;
       const float nmc = -(m_new * c);
-
-      if (j > 0) {       // GEMM 2 of the previous tile has read P_t and updated O_t
+      if (!__all_sync(0xFFFFFFFFu, o_ready)) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), abort_flag, p.status, 32));
         if (!ok) break;
-        tc_fence_after();
       }
+      tc_fence_after();
       TL(5)
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
+      // alpha = exp(m_old - m_new) (line 11) is exactly 1 for every row of a warp in which no maximum
+      // moved, so it is only evaluated on the rescaling path
+      float alpha = 1.0f;
 
       // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1.  Two
       // straight-line versions: the common one, and one that also rescales this thread's 64
@@ -525,11 +538,23 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       float l_tile = 0.0f;
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
+        if (kResc) alpha = ex2((m_old - m_new) * c);
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
-          const float pmax = ex2((bmax[b] - m_new) * c);
-          const int e = shared_exponent(__float_as_uint(pmax), kUos);
-          const float nb = nmc - (float)e;
+          // Shared exponent of the block from d = log2(pmax) = (bmax_b - m_new) * c <= 0, with no
+          // exponential: floor(log2 pmax) = floor(d), and the UOS rule raises the exponent iff the
+          // mantissa 2^(d - floor d) exceeds 1.8125, i.e. iff frac(d) > log2(1.8125).  d = 0 (the
+          // block holding the row maximum) gives e = -2 under both rules, as Appendix J derives.
+          // A block whose maximum underflows fp32 (d < -126, or fully masked) is a zero block.
+          const float d = (bmax[b] - m_new) * c;
+          const float rn = (d + 12582912.0f) - 12582912.0f;            // round to nearest integer
+          const float fl = rn > d ? rn - 1.0f : rn;                     // floor(d)
+          float ef = fl - 2.0f;
+          if (kUos && (d - fl) > 0.85798097f) ef += 1.0f;
+          ef = fmaxf(ef, -127.0f);
+          if (d < -126.0f) ef = 0.0f;
+          const int e = __float_as_int(ef + 12582912.0f) - 0x4B400000;  // exact small-integer conversion
+          const float nb = nmc - ef;
           uint4 w;
           float sx = 0.0f;
 #pragma unroll
