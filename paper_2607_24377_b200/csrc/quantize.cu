@@ -30,40 +30,25 @@ constexpr int kQThreads = 256;
 constexpr int kQUnroll = 4;
 
 // ------------------------------------------------------------------------------------------
-// Axis 1.  Work unit = one 16-byte chunk (8 elements).  `n_chunks` counts chunks of the OUTPUT
-// index space: for the canonical layout that is the input itself; for the tile layout rows are
-// padded to a multiple of 128 per matrix and padded rows read as zero.
-template <bool kTileLayout>
+// Axis 1, canonical layout: a linear streaming pass.  Work unit = one 16-byte chunk (8 elements);
+// chunk i yields code word i and (with its three neighbours) scale byte i / 4.
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
-                      uint8_t* __restrict__ scales, int64_t n_chunks, int64_t rows,
-                      int64_t rows_pad, bool uos) {
+                      uint8_t* __restrict__ scales, int64_t n_chunks, bool uos) {
   const int lane = threadIdx.x & 31;
   const int64_t stride = (int64_t)gridDim.x * kQThreads;
   // warp-uniform loop bound: every lane of a warp runs the same number of iterations
   const int64_t warp_first = (int64_t)blockIdx.x * kQThreads + (threadIdx.x & ~31);
   for (int64_t base = warp_first; base < n_chunks; base += stride * kQUnroll) {
     uint4 v[kQUnroll];
-    int64_t idx[kQUnroll];
 #pragma unroll
     for (int u = 0; u < kQUnroll; ++u) {
       const int64_t i = base + (int64_t)u * stride + lane;
-      idx[u] = i;
-      v[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (i < n_chunks) {
-        if (kTileLayout) {
-          const int64_t prow = i >> 4;               // padded global row (16 chunks per 128-wide row)
-          const int64_t b = prow / rows_pad;
-          const int64_t rr = prow - b * rows_pad;
-          if (rr < rows) v[u] = __ldg(in + ((b * rows + rr) << 4) + (i & 15));
-        } else {
-          v[u] = __ldg(in + i);
-        }
-      }
+      v[u] = i < n_chunks ? __ldg(in + i) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
     for (int u = 0; u < kQUnroll; ++u) {
-      const int64_t i = idx[u];
+      const int64_t i = base + (int64_t)u * stride + lane;
       uint32_t m = absmax_bf16x8(v[u]);
       m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
       m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
@@ -75,29 +60,58 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
       const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
       const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
       if (i >= n_chunks) continue;
-      if (kTileLayout) {
-        const int64_t prow = i >> 4;
-        const int64_t tile = prow >> 7;
-        const int r = (int)(prow & 127);
-        const int c = (int)((i >> 2) & 3);
-        codes[(tile * kTileCodeBytes + tile_code_offset(r, c)) / 4 + (i & 3)] = packed;
-        if ((lane & 15) == 0)
-          *reinterpret_cast<uint32_t*>(scales + tile * kTileScaleBytes + tile_scale_offset(r, 0)) =
-              eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
-      } else {
-        codes[i] = packed;
-        if ((lane & 15) == 0) {
-          const int64_t g = i >> 2;                  // block index, multiple of 4 here
-          if (i + 16 <= n_chunks) {
-            *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
-          } else {                                   // ragged end: fewer than 4 blocks left
-            scales[g] = (uint8_t)eb;
-            if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
-            if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
-          }
+      codes[i] = packed;
+      if ((lane & 15) == 0) {
+        const int64_t g = i >> 2;                    // block index, multiple of 4 here
+        if (i + 16 <= n_chunks) {
+          *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
+        } else {                                     // ragged end: fewer than 4 blocks left
+          scales[g] = (uint8_t)eb;
+          if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
+          if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
         }
       }
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Axis 1, tile layout (cols == 128).  grid = (row tiles, batch); one CTA quantizes one 128-row
+// tile: 32 KiB in, 8.5 KiB out.  A thread issues its eight 16-byte loads up front (the whole
+// tile is in flight at once), then quantizes them; a warp covers two full rows per step, so the
+// four lanes of a block and the sixteen lanes of a row are always in the same warp.
+__global__ void __launch_bounds__(kQThreads)
+quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
+                           uint8_t* __restrict__ scales, int64_t rows, bool uos) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t tile = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+  const int64_t row0 = (int64_t)blockIdx.x * kTile;
+  const uint4* src = in + ((int64_t)blockIdx.y * rows + row0) * 16;     // 16 chunks per row
+  const int rows_here = (int)min((int64_t)kTile, rows - row0);
+  uint4 v[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int chunk = k * kQThreads + tid;           // row = chunk >> 4
+    v[k] = (chunk >> 4) < rows_here ? __ldg(src + chunk) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  uint32_t* ctile = reinterpret_cast<uint32_t*>(codes + tile * kTileCodeBytes);
+  uint8_t* stile = scales + tile * kTileScaleBytes;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int chunk = k * kQThreads + tid;
+    const int r = chunk >> 4, c = (chunk >> 2) & 3;
+    uint32_t m = absmax_bf16x8(v[k]);
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+    const int e = shared_exponent(m << 16, uos);
+    const uint32_t packed = quantize_bf16x8(v[k], pow2_neg(e));
+    const uint32_t eb = (uint32_t)(e + 127);
+    const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
+    const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
+    const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
+    ctile[tile_code_offset(r, c) / 4 + (chunk & 3)] = packed;
+    if ((lane & 15) == 0)
+      *reinterpret_cast<uint32_t*>(stile + tile_scale_offset(r, 0)) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
   }
 }
 
@@ -213,12 +227,15 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
     const int64_t cap = 148 * 8 * 4;                       // a few waves of resident CTAs
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    if (tile)
-      quantize_axis1_kernel<true><<<(unsigned)blocks, kQThreads, 0, stream>>>(
-          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rows, rows_pad, uos);
-    else
-      quantize_axis1_kernel<false><<<(unsigned)blocks, kQThreads, 0, stream>>>(
-          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rows, rows_pad, uos);
+    if (tile) {
+      if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
+      dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
+      quantize_axis1_tile_kernel<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
+                                                                 (uint8_t*)scales, rows, uos);
+    } else {
+      quantize_axis1_kernel<<<(unsigned)blocks, kQThreads, 0, stream>>>(
+          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
+    }
   } else {
     const int64_t ct = (cols + kTile - 1) / kTile, rt = rows_pad / kTile;
     if (rt > 65535 || batch > 65535) return MXATTN_EUNSUPPORTED;
