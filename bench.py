@@ -234,14 +234,10 @@ def main():
     if rank == 0:
         sampler.stop()
     assert int(status[0].item()) == 0, "a bounded device-side wait expired"
-    total_ms = t_start.elapsed_time(t_stop)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
+    from paper_2607_24377_b200 import sharding
     flops = cfg.flops
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value, ms_per_step = sharding.aggregate_throughput(flops, t_start.elapsed_time(t_stop) / args.steps, world, "cuda")
+    value /= 1e12
 
     kern_ms = [float(np.mean([evs[i][a].elapsed_time(evs[i][a + 1]) for i in range(args.steps)])) for a in range(4)]
     attn_ms = kern_ms[3]
@@ -279,8 +275,7 @@ def main():
         for _ in range(n_e2e):
             mx.forward_host(hq, hk, hv, ho, B, H, Nq, Nkv, d, scale, flags, arena)   # synchronizes internally
         dt = (time.perf_counter() - t0) / n_e2e
-        if world > 1:
-            t = torch.tensor([dt], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); dt = float(t.item())
+        dt = sharding.max_over_ranks(dt, "cuda")
         e2e = {"value": world * flops / dt / 1e12, "unit": UNIT, "ms_per_step": dt * 1e3,
                "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
                "d2h_bytes_per_step": int(ho.numel()) * 2, "steps": n_e2e}
@@ -299,6 +294,8 @@ def main():
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
                         "seconds": dt}
 
+    clocks = sampler.summary()
+    mufu_ceiling = 16 * 512 * 148 * clocks["sm_mhz"] * 1e6 / 1e12 if clocks.get("sm_mhz") else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -306,12 +303,15 @@ def main():
         "config": {"workload": cfg.name, "B": B, "H": H, "Nq": Nq, "Nkv": Nkv, "d": d, "flags": "uos|pnq",
                    "out": "bf16", "l2": "inputs (2.3 GB at wan22) exceed L2; no flush needed",
                    "sharding": "one full batch per GPU, no collective"},
-        "clocks": sampler.summary(),
+        "clocks": clocks,
         "e2e": e2e, "gpu_launches": 4 * args.steps,
         "roofline": {"bound": "tensor", "kernel": "attention_kernel<uos,pnq>", "achieved": attn_tflops,
                      "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak, "traffic": None,
                      "peak_note": f"dense FP4 = {peaks['source']} sustained bf16 cuBLAS {peaks['bf16_tflops_sustained']} x nominal ratio 4 (of {peaks['source']})",
-                     "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms},
+                     "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms,
+                     # the softmax exponentials bind before the tensor pipe does: 16 ex2 per clock per SM,
+                     # one per (query, key) pair, 512 tensor flops per pair
+                     "mufu_ceiling_tflops": mufu_ceiling, "frac_of_mufu_ceiling": attn_tflops / mufu_ceiling if mufu_ceiling else None},
         "cpu_baseline": cpu_baseline,
         "kernels_ms": {"quantize_q": kern_ms[0], "quantize_k": kern_ms[1], "quantize_v": kern_ms[2], "attention": attn_ms},
         "quantize": quant, "variants": variants,
