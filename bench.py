@@ -31,6 +31,10 @@ UNIT = "TFLOP/s"
 NOMINAL_FP4_TFLOPS = 9000.0      # dense FP4, nominal
 FP4_OVER_BF16 = 4.0              # nominal ratio of dense FP4 to dense bf16 tensor throughput
 QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0
+# DRAM bytes of one attention launch, from the ncu capture of the same kernel on sweep16384
+# (256.7 MB, profiles/attention_kernel_sweep16384.txt) scaled by tokens x heads (traffic follows the
+# operand bytes, not the flops).
+ATTN_TRAFFIC_PER_TOKEN_HEAD = 256.7e6 / (16384 * 40)
 
 
 def load_peaks():
@@ -306,7 +310,9 @@ def main():
         "clocks": clocks,
         "e2e": e2e, "gpu_launches": 4 * args.steps,
         "roofline": {"bound": "tensor", "kernel": "attention_kernel<uos,pnq>", "achieved": attn_tflops,
-                     "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak, "traffic": None,
+                     "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak,
+                     "traffic": ATTN_TRAFFIC_PER_TOKEN_HEAD * Nkv * B * H,
+                     "traffic_note": "ncu dram bytes of a sweep16384 launch scaled by tokens x heads",
                      "peak_note": f"dense FP4 = {peaks['source']} sustained bf16 cuBLAS {peaks['bf16_tflops_sustained']} x nominal ratio 4 (of {peaks['source']})",
                      "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms,
                      # the softmax exponentials bind before the tensor pipe does: 16 ex2 per clock per SM,

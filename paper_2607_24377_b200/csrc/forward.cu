@@ -19,17 +19,20 @@
 //
 // Per KV tile a softmax thread (Algorithm 2 lines 10-14, for its half row):
 //   reads its 64 scores from tensor memory, takes its two 32-block maxima, exchanges the half-row
-//   maximum with its partner thread through shared memory, m_new = max(m, rowmax),
-//   alpha = exp(m - m_new);  for each of its blocks b:
-//     pmax  = exp2((bmax_b - m_new) * c)        -> shared exponent e_b by the UOS / OCP rule
+//   maximum with its partner thread through shared memory (64-thread named barrier),
+//   m_new = max(m, rowmax);  for each of its blocks b, with c = softmax_scale * log2 e:
+//     d     = (bmax_b - m_new) * c  = log2 of the block's largest exponential (<= 0)
+//     e_b   = floor(d) - 2, plus one under UOS when frac(d) > log2 1.8125      (no exponential needed:
+//             floor(log2 pmax) = floor(d), and the mantissa of pmax is 2^frac(d))
 //     x     = exp2(s * c - (m_new * c + e_b))   == P~ / 2^e_b   (the block scale folded into the exponent)
 //     codes = RNE-to-E2M1(x), 16 bytes, written into the K-major, 64B-swizzled A-operand tile
-//   and its two scale bytes into the scale-factor atom (c = softmax_scale * log2 e).  The
-//   difference (bmax_b - m_new) is formed exactly first, so the block holding the row maximum sees
-//   pmax = exp2(0) = 1 exactly and gets the scale the paper's Appendix J derives; the elements
-//   themselves take one fused multiply-add each.
-//   If m moved, the thread rescales its 64 accumulator columns in tensor memory by alpha
-//   (line 15); those tensor-memory round trips are interleaved with the exponentials.
+//   and its two scale bytes into the scale-factor atom.  The difference (bmax_b - m_new) is formed
+//   exactly first, so the block holding the row maximum has d = 0 and gets e = -2 under both rules,
+//   the scale the paper's Appendix J derives; the elements take one fused multiply-add and one
+//   ex2.approx each.
+//   If a row maximum of the warp moved, the thread rescales its 64 accumulator columns in tensor
+//   memory by alpha = exp(m - m_new) (line 15); those tensor-memory round trips are interleaved with
+//   the exponentials (the loop body exists in two straight-line versions).
 //
 // Tensor-memory map (512 columns): S [0,128) shared by both groups (each group copies its scores
 // to registers at once, so the buffer is free again long before the other group needs it),
@@ -60,7 +63,7 @@ constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
 constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
 constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
-constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2 + 1;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
+constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
 constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
@@ -134,10 +137,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
-#ifdef EXP_TIMELINE
-    if (code >= 31 && blockIdx.x == 300 && (threadIdx.x == 0 || threadIdx.x == 256)) atomicAdd(status + 8 + (code - 31) + 4 * (threadIdx.x >> 8), 1);
-    if (code < 31 && blockIdx.x == 300) atomicAdd(status + 4000 + code, 1);
-#endif
     if (mbar_try(bar, parity)) return true;
     if ((it & 15) == 0) {
       if (*abort_flag) return false;
@@ -248,8 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
     }
     mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-    mbar_init(bar(BAR_SFREE), 8);
-    mbar_init(bar(kNumBars - 1), 8);
+    mbar_init(bar(BAR_SFREE), 8);                  // one arrival per softmax warp of the draining group
     mbar_init(bar(BAR_PFULL + 0), 8); mbar_init(bar(BAR_PFULL + 1), 8);   // one arrival per softmax warp
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
     *abort_flag = 0;
@@ -361,47 +359,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         tc_cp_sf(tmem + kColSFV + 4, sbase + kOffSFOnes);        // scales of the ones rows, both slots
         tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
       }
-#ifdef EXP_TWO_S
-      auto gemm1x = [&](int t, int j) {
-        const int s = j % kStages;
-#pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
-          const uint64_t da = make_desc(sbase + kOffQ + t * kTileCodeBytes + ks * 32, 512, 4);
-          const uint64_t db = make_desc(sbase + kOffK + s * kTileCodeBytes + ks * 32, 512, 4);
-          tc_mma(tmem + kColS + 128 * t, da, db, make_idesc(128, ks), tmem + kColSFQ + 4 * t, tmem + kColSFK + 4 * (j & 1), ks);
-        }
-        tc_commit(bar(BAR_SFULL + t));
-      };
-      ok = ok && wait_k(0);
-      if (ok) { gemm1x(0, 0); gemm1x(1, 0); tc_commit(bar(BAR_KEMPTY + 0)); }
-      for (int j = 0; j < T && ok; ++j) {
-        const int s = j % kStages;
-        if (j + 1 < T) {
-          ok = wait_k(j + 1);
-          ok = ok && mbar_wait(bar(BAR_SFREE), (uint32_t)(j & 1), abort_flag, p.status, 23);
-          if (!ok) break;
-          tc_fence_after();
-          gemm1x(0, j + 1);
-          ok = mbar_wait(bar(kNumBars - 1), (uint32_t)(j & 1), abort_flag, p.status, 23);
-          if (!ok) break;
-          tc_fence_after();
-          gemm1x(1, j + 1);
-          tc_commit(bar(BAR_KEMPTY + (j + 1) % kStages));
-        }
-        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);
-        ok = ok && mbar_wait(bar(BAR_VFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 25);
-        if (!ok) break;
-        tc_fence_after();
-        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
-        gemm2(0, j);
-        ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
-        if (!ok) break;
-        tc_fence_after();
-        gemm2(1, j);
-        tc_commit(bar(BAR_VEMPTY + s));
-      }
-    }
-#else
       // prologue: S(0,0), S(1,0), S(0,1)
       ok = ok && wait_k(0);
       if (ok) gemm1(0, 0);
@@ -439,18 +396,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       }
     }
-#endif
   } else if (warp < kSoftmaxWarps) {
     // =============================== softmax groups =========================================
     const int t = warp >> 3;                       // query tile of this group
     const int h = (warp >> 2) & 1;                 // which 64 key columns of the tile
     const int row = (warp & 3) * 32 + lane;        // row within the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-#ifdef EXP_TWO_S
-    const uint32_t t_s = tmem + kColS + 128 * t + lane_addr + 64 * h;
-#else
     const uint32_t t_s = tmem + kColS + lane_addr + 64 * h;
-#endif
     const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;     // column 0 of this row's accumulator
     const float c = p.scale_log2e;
     float m_run = -INFINITY;
@@ -461,30 +413,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
     bool ok = true;
 
-#ifdef EXP_TIMELINE
-#define TL(k) if (blockIdx.x == 300 && lane == 0 && (warp == 0 || warp == 8 || warp == 4) && j >= 40 && j < 48) \
-    reinterpret_cast<long long*>(p.status + 16)[((warp >> 2) * 8 + (j - 40)) * 8 + (k)] = clock64();
-#else
-#define TL(k)
-#endif
     for (int j = 0; j < T; ++j) {
-      TL(0)
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
       TMEM_LD32(t_s + 0, (sr + 0));
       TMEM_LD32(t_s + 32, (sr + 32));
-      TL(1)
       tmem_ld_wait();
-      TL(2)
       tc_fence_before();
       __syncwarp();
-#ifdef EXP_TWO_S
-      if (lane == 0) mbar_arrive(bar(t ? kNumBars - 1 : BAR_SFREE));
-#else
       if (lane == 0) mbar_arrive(bar(BAR_SFREE));  // the score buffer may be overwritten
-#endif
 
       if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
         const int valid = (int)(p.Nkv - (int64_t)j * kTile) - 64 * h;
@@ -512,9 +451,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t
       // or rescales O_t; probe that barrier now so its latency overlaps the pair barrier
       const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
-      TL(3)
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
-      TL(4)
       const float m_new = max3(m_run, fmaxf(bmax[0], bmax[1]), mslot[(h ^ 1) * 128 + row]);        // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
@@ -525,7 +462,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         if (!ok) break;
       }
       tc_fence_after();
-      TL(5)
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
       // alpha = exp(m_old - m_new) (line 11) is exactly 1 for every row of a warp in which no maximum
       // moved, so it is only evaluated on the rescaling path
@@ -591,14 +527,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       };
       if (rescale) tile_body(std::true_type{}); else tile_body(std::false_type{});
-      TL(6)
       *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
-      TL(7)
     }
 
     // ---- epilogue: O = O~ / l (line 18) ----
