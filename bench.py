@@ -266,6 +266,24 @@ def main():
             ms = a.elapsed_time(b) / n
             variants[name] = {"attn_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12}
         variants["uos_pnq_over_ocp_direct_time"] = variants["uos_pnq"]["attn_ms"] / variants["ocp_direct"]["attn_ms"]
+        # bf16 reference point: NOT a kernel of this repository -- PyTorch's fused SDPA (library flash /
+        # cuDNN attention) on the same bf16 tensors.  A bf16 (kind::f16) variant of this repo's own
+        # kernel is not built yet.
+        try:
+            import torch.nn.functional as F
+            ob = F.scaled_dot_product_attention(dq, dk, dv, scale=scale); del ob
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(2):
+                ob = F.scaled_dot_product_attention(dq, dk, dv, scale=scale)
+            b.record(); torch.cuda.synchronize(); del ob
+            ms = a.elapsed_time(b) / 2
+            variants["bf16_library_sdpa"] = {"attn_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                                             "note": "torch.nn.functional.scaled_dot_product_attention, library kernel, context only"}
+            variants["uos_pnq_speedup_over_bf16_library"] = ms / variants["uos_pnq"]["attn_ms"]
+        except Exception as exc:  # pragma: no cover
+            variants["bf16_library_sdpa"] = {"unavailable": str(exc)[:200]}
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
