@@ -266,6 +266,18 @@ def main():
             ms = a.elapsed_time(b) / n
             variants[name] = {"attn_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12}
         variants["uos_pnq_over_ocp_direct_time"] = variants["uos_pnq"]["attn_ms"] / variants["ocp_direct"]["attn_ms"]
+        # Algorithm 2 lines 1-2 fused into the Q/K quantize launches (the attention launch is unchanged)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        rot = mx.MODE_UOS | mx.MODE_HADAMARD
+        mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, rot, mx.LAYOUT_TILE); torch.cuda.synchronize()
+        a.record()
+        for _ in range(3):
+            mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, rot, mx.LAYOUT_TILE)
+        b.record(); torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 3
+        variants["quantize_q_with_hadamard"] = {"ms": ms, "GBps": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9,
+                                                "frac_of_hbm_peak": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, mx.MODE_UOS, mx.LAYOUT_TILE)       # restore the unrotated Q-hat
         # bf16 reference point: NOT a kernel of this repository -- PyTorch's fused SDPA (library flash /
         # cuDNN attention) on the same bf16 tensors.  A bf16 (kind::f16) variant of this repo's own
         # kernel is not built yet.

@@ -38,14 +38,25 @@ extern "C" {
  * M is the largest magnitude in the block; an all-zero block gets sigma = 1 (byte 127) and
  * all-zero codes; e is clamped to [-127, 127]. */
 typedef enum { MXATTN_MODE_OCP = 0, MXATTN_MODE_UOS = 1 } mxattn_mode;
+/* OR-able into `mode` of the quantizer: first apply the fixed orthogonal Hadamard rotation
+ * y = x H_128 / sqrt(128) to every row (paper Algorithm 2, lines 1-2; Section 4.3), then quantize y.
+ * H_128 is the Sylvester matrix, H[i][j] = (-1)^popcount(i & j).  The rotation is evaluated in fp32
+ * as the fast Walsh-Hadamard butterfly with strides 1, 2, ..., 64, each stage (a, b) -> (a + b, a - b),
+ * followed by one multiply by fl32(1/sqrt(128)); there is no rounding to bf16 in between.
+ * Only block_axis 1 with cols == 128. */
+enum { MXATTN_MODE_HADAMARD = 0x100 };
 
 /* Flags of the forward pass.
  * UOS      : use the UOS rule for Q, K, V and the softmax tiles (else the OCP rule for all four).
  * PNQ      : the row sum l is accumulated from the QUANTIZED exponentials (paper Eq. 22,
  *            Algorithm 2 line 14); without it l is accumulated from the unquantized ones
  *            (the "direct" placement, paper Eq. 12).
- * OUT_FP32 : `o` is fp32 instead of bf16. */
-enum { MXATTN_FLAG_UOS = 1, MXATTN_FLAG_PNQ = 2, MXATTN_FLAG_OUT_FP32 = 4 };
+ * OUT_FP32 : `o` is fp32 instead of bf16.
+ * HADAMARD : see below. */
+enum { MXATTN_FLAG_UOS = 1, MXATTN_FLAG_PNQ = 2, MXATTN_FLAG_OUT_FP32 = 4,
+       /* rotate Q and K with the fixed Hadamard matrix before quantizing them (Algorithm 2 lines 1-2);
+        * Q K^T is unchanged by the rotation in exact arithmetic, the quantization error is not */
+       MXATTN_FLAG_HADAMARD = 8 };
 
 typedef enum {
   MXATTN_OK = 0,

@@ -15,7 +15,7 @@ Per head and per query row (rows are independent; the query tile size never ente
         m      = m_new                                                 (line 16)
     O = O~ / l                                                         (line 18)
 
-The Hadamard rotation of lines 1-2 is outside this hot path.  The same scale rule (UOS or the
+The Hadamard rotation of lines 1-2 is optional (`rotate`).  The same scale rule (UOS or the
 OCP floor rule) is used for all four tensors Q, K, V and P~ (Section 4.3; the "MXFP4 (OCP)"
 baseline of Section 5.2).  float64 everywhere except the single fp32 rounding of P~, which is
 the precision in which the quantizer sees the exponentials.
@@ -33,8 +33,12 @@ from . import mxfp4
 B_C = 128
 
 
-def quantize_qkv(q, k, v, rule):
-    """Dequantized Q-hat, K-hat, V-hat (float64) of one head. q [Nq,d], k,v [Nkv,d]."""
+def quantize_qkv(q, k, v, rule, rotate: bool = False):
+    """Dequantized Q-hat, K-hat, V-hat (float64) of one head. q [Nq,d], k,v [Nkv,d].
+    rotate: apply the fixed Hadamard rotation to Q and K first (Algorithm 2 lines 1-2)."""
+    if rotate:
+        q = mxfp4.hadamard_rotate_f32(q)
+        k = mxfp4.hadamard_rotate_f32(k)
     qd = mxfp4.quantize_dequantize(q, axis=1, rule=rule)
     kd = mxfp4.quantize_dequantize(k, axis=1, rule=rule)
     vd = mxfp4.quantize_dequantize(v, axis=0, rule=rule)
@@ -43,7 +47,7 @@ def quantize_qkv(q, k, v, rule):
 
 def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True,
                  rows=None, quantize_inputs: bool = True, quantize_p: bool = True,
-                 return_state: bool = False):
+                 return_state: bool = False, rotate: bool = False):
     """Algorithm 2 for one head.
 
     q [Nq,d], k [Nkv,d], v [Nkv,d]: float arrays holding bf16-representable values.
@@ -58,7 +62,7 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     if quantize_inputs:
-        qd, kd, vd = quantize_qkv(q, k, v, rule)
+        qd, kd, vd = quantize_qkv(q, k, v, rule, rotate)
     else:
         qd, kd, vd = q, k, v
     if rows is not None:
@@ -102,14 +106,14 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     return out
 
 
-def forward(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True):
+def forward(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True, rotate: bool = False):
     """All heads. q [B,H,Nq,d], k,v [B,H,Nkv,d] -> O [B,H,Nq,d] float64."""
     q = np.asarray(q)
     B, H = q.shape[:2]
     out = np.empty(q.shape, dtype=np.float64)
     for b in range(B):
         for h in range(H):
-            out[b, h] = forward_head(q[b, h], k[b, h], v[b, h], softmax_scale, uos, pnq)
+            out[b, h] = forward_head(q[b, h], k[b, h], v[b, h], softmax_scale, uos, pnq, rotate=rotate)
     return out
 
 

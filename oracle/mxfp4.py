@@ -150,3 +150,35 @@ def quantize_matrix_canonical(x: np.ndarray, block_axis: int, rule: ScaleRule):
         codes, e = quantize_blocks(xt.reshape(cols, rows_pad // BLOCK, BLOCK), rule)
         return pack_nibbles(codes.reshape(cols, rows_pad)), e8m0_bytes(e)
     raise ValueError(block_axis)
+
+
+# ----------------------------------------------------------------------------- Hadamard rotation
+def hadamard_matrix(n: int) -> np.ndarray:
+    """Sylvester Hadamard matrix H_n (n a power of two): H[i, j] = (-1)^popcount(i & j), entries +-1."""
+    i = np.arange(n)
+    bits = i[:, None] & i[None, :]
+    pop = np.zeros_like(bits)
+    while bits.any():
+        pop += bits & 1
+        bits >>= 1
+    return np.where(pop % 2 == 0, 1.0, -1.0)
+
+
+def hadamard_rotate_f32(x: np.ndarray) -> np.ndarray:
+    """x R_H along the last axis with R_H = H_n / sqrt(n) (Algorithm 2 lines 1-2: the fixed orthogonal
+    Hadamard rotation), evaluated in fp32 the way the quantizer sees it: the fast Walsh-Hadamard
+    butterfly with strides 1, 2, 4, ..., n/2, each stage (a, b) -> (a + b, a - b) in IEEE fp32, then one
+    fp32 multiply by fl32(1/sqrt(n)).  Returns fp32.  (The precision and the stage order are part of
+    the definition because the result feeds a rounding decision.)"""
+    y = np.array(x, dtype=np.float32, copy=True)
+    n = y.shape[-1]
+    assert n & (n - 1) == 0
+    stride = 1
+    while stride < n:
+        v = y.reshape(y.shape[:-1] + (n // (2 * stride), 2, stride))
+        a = v[..., 0, :].copy()
+        b = v[..., 1, :].copy()
+        v[..., 0, :] = a + b
+        v[..., 1, :] = a - b
+        stride *= 2
+    return y * np.float32(1.0 / np.sqrt(np.float64(n)))

@@ -5,7 +5,7 @@ The compute lives in ``libmxattn.so`` (hand-written sm_100a CUDA behind a C ABI,
 fallback and raises if the library is missing.
 """
 from .binding import (  # noqa: F401
-    FLAG_OUT_FP32, FLAG_PNQ, FLAG_UOS, LAYOUT_CANONICAL, LAYOUT_TILE, MODE_OCP, MODE_UOS,
+    FLAG_HADAMARD, FLAG_OUT_FP32, FLAG_PNQ, FLAG_UOS, LAYOUT_CANONICAL, LAYOUT_TILE, MODE_HADAMARD, MODE_OCP, MODE_UOS,
     MxAttnError, device_status, forward, forward_host, forward_host_arena_bytes, forward_prequantized,
     forward_static, forward_workspace_bytes, forward_ws, last_launch_count, lib, lib_path, quantize_mxfp4,
     quantize_mxfp4_batched, set_workspace, strerror,

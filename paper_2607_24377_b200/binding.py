@@ -12,8 +12,8 @@ import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 
-MODE_OCP, MODE_UOS = 0, 1
-FLAG_UOS, FLAG_PNQ, FLAG_OUT_FP32 = 1, 2, 4
+MODE_OCP, MODE_UOS, MODE_HADAMARD = 0, 1, 0x100
+FLAG_UOS, FLAG_PNQ, FLAG_OUT_FP32, FLAG_HADAMARD = 1, 2, 4, 8
 LAYOUT_CANONICAL, LAYOUT_TILE = 0, 1
 
 _lib = None

@@ -38,7 +38,7 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
                       size_t workspace_bytes, cudaStream_t stream) {
   if (!q || !k || !v || !o) return MXATTN_EINVAL;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
-  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32 | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
   if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
   if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return MXATTN_EALIGN;
@@ -49,12 +49,13 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
   g_launches = 0;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   const int mode = (flags & MXATTN_FLAG_UOS) ? MXATTN_MODE_UOS : MXATTN_MODE_OCP;
+  const int qk_mode = mode | ((flags & MXATTN_FLAG_HADAMARD) ? MXATTN_MODE_HADAMARD : 0);   // Algorithm 2 lines 1-2
   const int64_t bh = (int64_t)B * H;
   if (cudaMemsetAsync(ws + w.status, 0, 16, stream) != cudaSuccess) return MXATTN_ECUDA;
   int rc;
   // Algorithm 2 lines 3-5: Q-hat, K-hat (blocks along d), V-hat (blocks along tokens)
-  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
-  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
   if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
   // lines 6-19
   return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
@@ -98,7 +99,7 @@ extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_sc
                                            float softmax_scale, unsigned flags, void* status, void* stream) {
   if (!q_codes || !q_scales || !k_codes || !k_scales || !v_codes || !v_scales || !o || !status) return MXATTN_EINVAL;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
-  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32 | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
   if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
   if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
   if (!aligned16(q_codes) || !aligned16(q_scales) || !aligned16(k_codes) || !aligned16(k_scales) ||

@@ -98,7 +98,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t sbo_bytes
 }
 
 // instruction descriptor of kind::mxf4.block_scale: A, B = E2M1 (K-major), scales UE8M0, M = 128
-__device__ __forceinline__ uint32_t make_idesc(int n, int ks) {
+__device__ __forceinline__ constexpr uint32_t make_idesc(int n, int ks) {
   return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
          ((uint32_t)(ks * 2) << 29) | ((uint32_t)(ks * 2) << 4);
 }
@@ -155,7 +155,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 }
 
 __device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint32_t saddr) {   // 512-byte scale atom -> 4 columns
-  const uint64_t d = make_desc(saddr, 128, 0);
+  const uint64_t d = ((uint64_t)((128u >> 4) | (1u << 14)) << 32) | (saddr >> 4);   // no swizzle, 8-row groups 128 B apart
   asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
 }
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -317,26 +317,29 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     if (lane == 0) {
       bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag, p.status, 21);
       uint32_t sfree_n = 0;      // completed phases of S_FREE consumed so far
+      // Descriptor words are loop invariants up to a stage offset: the low word is the shared
+      // address >> 4 (all tiles sit below 256 KiB, so it fits the 14-bit field), the high word is
+      // constant (stride between 8-row groups, descriptor version, swizzle mode).
+      constexpr uint32_t kDescHiTile = (512u >> 4) | (1u << 14) | (4u << 29);   // 64-byte swizzle, K-major
+      const uint32_t q_lo = (sbase + kOffQ) >> 4, k_lo = (sbase + kOffK) >> 4;
+      const uint32_t v_lo = (sbase + kOffV) >> 4, p_lo = (sbase + kOffP) >> 4;
+      auto desc = [](uint32_t lo) { return ((uint64_t)kDescHiTile << 32) | lo; };
       auto gemm1 = [&](int t, int j) {      // S = Q_t K_j^T
-        const int s = j % kStages;
-#pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
-          const uint64_t da = make_desc(sbase + kOffQ + t * kTileCodeBytes + ks * 32, 512, 4);
-          const uint64_t db = make_desc(sbase + kOffK + s * kTileCodeBytes + ks * 32, 512, 4);
-          tc_mma(tmem + kColS, da, db, make_idesc(128, ks), tmem + kColSFQ + 4 * t, tmem + kColSFK + 4 * (j & 1), ks);
-        }
+        const uint32_t a = q_lo + (uint32_t)t * (kTileCodeBytes >> 4);
+        const uint32_t b = k_lo + (uint32_t)(j % kStages) * (kTileCodeBytes >> 4);
+        const uint32_t sfa = tmem + kColSFQ + 4 * t, sfb = tmem + kColSFK + 4 * (j & 1);
+        tc_mma(tmem + kColS, desc(a), desc(b), make_idesc(128, 0), sfa, sfb, 0u);
+        tc_mma(tmem + kColS, desc(a + 2), desc(b + 2), make_idesc(128, 1), sfa, sfb, 1u);   // K 64..127: +32 bytes
         tc_commit(bar(BAR_SFULL + t));
       };
       auto gemm2 = [&](int t, int j) {      // O_t += P_t [V_j | 1]
-        const int s = j % kStages;
         tc_cp_sf(tmem + kColSFP + 4 * t, sbase + kOffSFP + t * kTileScaleBytes);
-#pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
-          const uint64_t da = make_desc(sbase + kOffP + t * kTileCodeBytes + ks * 32, 512, 4);
-          const uint64_t db = make_desc(sbase + kOffV + s * kVStageBytes + ks * 32, 512, 4);
-          tc_mma(tmem + (t ? kColO1 : kColO0), da, db, make_idesc(kNV, ks), tmem + kColSFP + 4 * t,
-                 tmem + kColSFV + 8 * (j & 1), (j > 0 || ks > 0) ? 1u : 0u);
-        }
+        const uint32_t a = p_lo + (uint32_t)t * (kTileCodeBytes >> 4);
+        const uint32_t b = v_lo + (uint32_t)(j % kStages) * (kVStageBytes >> 4);
+        const uint32_t d = tmem + (t ? kColO1 : kColO0);
+        const uint32_t sfa = tmem + kColSFP + 4 * t, sfb = tmem + kColSFV + 8 * (j & 1);
+        tc_mma(d, desc(a), desc(b), make_idesc(kNV, 0), sfa, sfb, j > 0 ? 1u : 0u);
+        tc_mma(d, desc(a + 2), desc(b + 2), make_idesc(kNV, 1), sfa, sfb, 1u);
         tc_commit(bar(BAR_ODONE + t));
       };
       auto wait_k = [&](int j) {

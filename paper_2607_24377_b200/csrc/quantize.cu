@@ -26,12 +26,71 @@ __device__ __forceinline__ uint32_t quantize_bf16x8(const uint4& v, float inv) {
                      bf16lo(v.z) * inv, bf16hi(v.z) * inv, bf16lo(v.w) * inv, bf16hi(v.w) * inv);
 }
 
+// Fixed Hadamard rotation of one 128-element row held by 16 consecutive lanes, 8 elements per lane
+// (element index = 8 * (lane % 16) + i): y = x H_128 / sqrt(128) (paper Algorithm 2, lines 1-2).
+// Fast Walsh-Hadamard butterfly in fp32, strides 1, 2, 4 inside the thread and 8, 16, 32, 64 across
+// lanes, every stage (a, b) -> (a + b, a - b) with a the lower index, then one multiply by
+// fl32(1/sqrt(128)).  The stage order and the fp32 arithmetic are part of the definition, because
+// the result feeds a rounding decision; __fadd_rn / __fsub_rn keep the compiler from contracting.
+__device__ __forceinline__ void hadamard128_rows(float (&f)[8], int lane) {
+#pragma unroll
+  for (int s = 1; s < 8; s <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if ((i & s) == 0) {
+        const float a = f[i], b = f[i + s];
+        f[i] = __fadd_rn(a, b);
+        f[i + s] = __fsub_rn(a, b);
+      }
+    }
+  }
+#pragma unroll
+  for (int m = 1; m < 16; m <<= 1) {
+    const bool upper = (lane & m) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float other = __shfl_xor_sync(0xFFFFFFFFu, f[i], m);
+      f[i] = upper ? __fsub_rn(other, f[i]) : __fadd_rn(f[i], other);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) f[i] = __fmul_rn(f[i], 0.08838834764831845f);
+}
+
+// One 16-byte chunk (8 bf16) -> packed codes and the block's shared exponent; the four lanes of a
+// 32-element block combine their maxima with two shuffles.  With kRotate the 16 lanes of a row
+// first apply the Hadamard rotation and the block maximum is taken on the fp32 results.
+template <bool kRotate>
+__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, bool uos, int* e_out) {
+  if (kRotate) {
+    float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y), bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
+    hadamard128_rows(f, lane);
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = max(m, __float_as_uint(f[i]) & 0x7FFFFFFFu);
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+    const int e = shared_exponent(m, uos);
+    const float inv = pow2_neg(e);
+    *e_out = e;
+    return pack_e2m1x8(f[0] * inv, f[1] * inv, f[2] * inv, f[3] * inv, f[4] * inv, f[5] * inv, f[6] * inv, f[7] * inv);
+  } else {
+    uint32_t m = absmax_bf16x8(v);
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+    const int e = shared_exponent(m << 16, uos);
+    *e_out = e;
+    return quantize_bf16x8(v, pow2_neg(e));
+  }
+}
+
 constexpr int kQThreads = 256;
 constexpr int kQUnroll = 4;
 
 // ------------------------------------------------------------------------------------------
 // Axis 1, canonical layout: a linear streaming pass.  Work unit = one 16-byte chunk (8 elements);
 // chunk i yields code word i and (with its three neighbours) scale byte i / 4.
+template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t n_chunks, bool uos) {
@@ -49,11 +108,8 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
 #pragma unroll
     for (int u = 0; u < kQUnroll; ++u) {
       const int64_t i = base + (int64_t)u * stride + lane;
-      uint32_t m = absmax_bf16x8(v[u]);
-      m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-      m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-      const int e = shared_exponent(m << 16, uos);
-      const uint32_t packed = quantize_bf16x8(v[u], pow2_neg(e));
+      int e;
+      const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, uos, &e);
       // four consecutive blocks (16 lanes) -> one 32-bit scale word
       const uint32_t eb = (uint32_t)(e + 127);
       const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
@@ -80,6 +136,7 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
 // tile: 32 KiB in, 8.5 KiB out.  A thread issues its eight 16-byte loads up front (the whole
 // tile is in flight at once), then quantizes them; a warp covers two full rows per step, so the
 // four lanes of a block and the sixteen lanes of a row are always in the same warp.
+template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
                            uint8_t* __restrict__ scales, int64_t rows, bool uos) {
@@ -100,11 +157,8 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
   for (int k = 0; k < 8; ++k) {
     const int chunk = k * kQThreads + tid;
     const int r = chunk >> 4, c = (chunk >> 2) & 3;
-    uint32_t m = absmax_bf16x8(v[k]);
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-    const int e = shared_exponent(m << 16, uos);
-    const uint32_t packed = quantize_bf16x8(v[k], pow2_neg(e));
+    int e;
+    const uint32_t packed = quantize_chunk<kRotate>(v[k], lane, uos, &e);
     const uint32_t eb = (uint32_t)(e + 127);
     const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
     const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
@@ -211,7 +265,10 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
   if (!in || !codes || !scales) return MXATTN_EINVAL;
   if (batch <= 0 || rows <= 0 || cols <= 0) return MXATTN_EINVAL;
   if (block_axis != 0 && block_axis != 1) return MXATTN_EINVAL;
+  const bool rotate = (mode & MXATTN_MODE_HADAMARD) != 0;
+  mode &= ~MXATTN_MODE_HADAMARD;
   if (mode != MXATTN_MODE_OCP && mode != MXATTN_MODE_UOS) return MXATTN_EINVAL;
+  if (rotate && (block_axis != 1 || cols != kHeadDim)) return MXATTN_EUNSUPPORTED;
   if (layout != MXATTN_LAYOUT_CANONICAL && layout != MXATTN_LAYOUT_TILE) return MXATTN_EINVAL;
   if (layout == MXATTN_LAYOUT_TILE && cols != kHeadDim) return MXATTN_EUNSUPPORTED;
   if (block_axis == 1 && cols % kBlock != 0) return MXATTN_EUNSUPPORTED;
@@ -230,11 +287,19 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
     if (tile) {
       if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
-      quantize_axis1_tile_kernel<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
-                                                                 (uint8_t*)scales, rows, uos);
+      if (rotate)
+        quantize_axis1_tile_kernel<true><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
+                                                                         (uint8_t*)scales, rows, uos);
+      else
+        quantize_axis1_tile_kernel<false><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
+                                                                          (uint8_t*)scales, rows, uos);
     } else {
-      quantize_axis1_kernel<<<(unsigned)blocks, kQThreads, 0, stream>>>(
-          (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
+      if (rotate)
+        quantize_axis1_kernel<true><<<(unsigned)blocks, kQThreads, 0, stream>>>(
+            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
+      else
+        quantize_axis1_kernel<false><<<(unsigned)blocks, kQThreads, 0, stream>>>(
+            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
     }
   } else {
     const int64_t ct = (cols + kTile - 1) / kTile, rt = rows_pad / kTile;

@@ -15,10 +15,11 @@ REL_L2_TOL = 1e-3      # the tolerance the benchmark spec states for the fp32 output
 MAX_ABS_TOL = 4e-3
 
 
-def run_forward(cfg, q, k, v, uos, pnq, f32=True):
+def run_forward(cfg, q, k, v, uos, pnq, f32=True, rotate=False):
     import paper_2607_24377_b200 as mx
     dq, dk, dv = util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v)
-    flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | (mx.FLAG_OUT_FP32 if f32 else 0)
+    flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | (mx.FLAG_OUT_FP32 if f32 else 0) | \
+            (mx.FLAG_HADAMARD if rotate else 0)
     out = torch.full((cfg.B, cfg.H, cfg.Nq, cfg.d), float("nan"), dtype=torch.float32 if f32 else torch.bfloat16, device="cuda")
     ws = torch.empty(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), dtype=torch.uint8, device="cuda")
     mx.forward_ws(dq, dk, dv, out, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, flags, ws)
@@ -27,9 +28,9 @@ def run_forward(cfg, q, k, v, uos, pnq, f32=True):
     return out
 
 
-def oracle_out(cfg, q, k, v, uos, pnq):
+def oracle_out(cfg, q, k, v, uos, pnq, rotate=False):
     f = util.bits_to_f64
-    return attention.forward(f(q), f(k), f(v), cfg.softmax_scale, uos, pnq)
+    return attention.forward(f(q), f(k), f(v), cfg.softmax_scale, uos, pnq, rotate=rotate)
 
 
 def check(got, want):
@@ -114,3 +115,20 @@ def test_host_buffer_entry_point():
     arena = torch.empty(mx.forward_host_arena_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, flags), dtype=torch.uint8, device="cuda")
     mx.forward_host(hq, hk, hv, ho, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, cfg.softmax_scale, flags, arena)
     assert torch.equal(ho, want)
+
+
+@pytest.mark.parametrize("recipe", ["iid", "outlier", "wan"])
+def test_full_algorithm_with_hadamard_rotation(recipe):
+    # Algorithm 2 complete: lines 1-2 (rotation of Q and K) fused into the quantize launches
+    cfg = si.custom_config("rot", 1, 2, 300, 1000, 91, recipe)
+    q, k, v = si.make_all(cfg)
+    got = run_forward(cfg, q, k, v, True, True, rotate=True)
+    want = oracle_out(cfg, q, k, v, True, True, rotate=True)
+    check(got, want)
+    if recipe != "iid":     # and it is the better approximation of float64 dense attention on outlier data
+        f = util.bits_to_f64
+        dense = np.stack([attention.dense_attention_head(f(q[0, h]), f(k[0, h]), f(v[0, h]), cfg.softmax_scale) for h in range(2)])[None]
+        plain = run_forward(cfg, q, k, v, True, True).double().cpu().numpy()
+        e_rot = np.linalg.norm(got.double().cpu().numpy() - dense) / np.linalg.norm(dense)
+        e_plain = np.linalg.norm(plain - dense) / np.linalg.norm(dense)
+        assert e_rot < e_plain

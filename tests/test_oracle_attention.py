@@ -215,3 +215,21 @@ def test_all_heads_wrapper():
     out = attention.forward(f(q), f(k), f(v), SCALE)
     assert out.shape == (1, 2, 64, 128)
     assert np.allclose(out[0, 1], attention.forward_head(f(q)[0, 1], f(k)[0, 1], f(v)[0, 1], SCALE), rtol=0, atol=1e-13)
+
+
+def test_rotation_brings_the_quantized_output_closer_to_dense_attention_on_outlier_data():
+    # Table 3 of the paper attributes the largest quality gain to the Hadamard rotation; on synthetic
+    # channel-outlier data the ordering must at least hold
+    q, k, v = head(256, 1024, 23, "outlier")
+    dense = attention.dense_attention_head(q, k, v, SCALE)
+    plain = rel_l2(attention.forward_head(q, k, v, SCALE, True, True), dense)
+    rot = rel_l2(attention.forward_head(q, k, v, SCALE, True, True, rotate=True), dense)
+    assert rot < plain
+
+
+def test_rotation_with_identity_quantizer_changes_nothing():
+    q, k, v = head(32, 256, 24)
+    rq = mxfp4.hadamard_rotate_f32(q).astype(np.float64); rk = mxfp4.hadamard_rotate_f32(k).astype(np.float64)
+    a = attention.forward_head(rq, rk, v, SCALE, quantize_inputs=False, quantize_p=False)
+    b = attention.dense_attention_head(q, k, v, SCALE)
+    assert np.abs(a - b).max() < 1e-5

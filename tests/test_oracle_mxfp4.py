@@ -293,3 +293,39 @@ def test_canonical_packing_layouts():
     assert sc[5, 1] == 126 and codes[5, 16] == ((7 | 8) << 4)   # token 33 -> byte 16 high nibble; -3/0.5 = -6
     assert sc[31, 1] == 124 and codes[31, 19] == (6 << 4)       # 0.5 / 2^-3 = 4, token 39
     assert np.all(sc[:, 2:] == 127) and np.all(codes[:, 20:] == 0)
+
+
+# ---------------------------------------------------------------- Hadamard rotation (Algorithm 2 lines 1-2)
+def test_hadamard_matrix_is_the_sylvester_construction():
+    h2 = np.array([[1, 1], [1, -1]], dtype=np.float64)
+    h = h2
+    for _ in range(6):
+        h = np.kron(h2, h)                                   # textbook recursion H_2n = H_2 (x) H_n
+    assert np.array_equal(mxfp4.hadamard_matrix(128), h)
+    assert np.array_equal(h @ h.T, 128 * np.eye(128))        # orthogonal up to the factor n
+
+
+def test_fast_rotation_equals_matrix_product_and_is_orthogonal():
+    rng = np.random.default_rng(8)
+    x = bf16_bits_to_f32(__import__("synth_inputs").f32_to_bf16_bits(rng.standard_normal((300, 128)).astype(np.float32)))
+    x[::7, 5] *= 16
+    y = mxfp4.hadamard_rotate_f32(x).astype(np.float64)
+    want = x.astype(np.float64) @ (mxfp4.hadamard_matrix(128) / np.sqrt(128.0))
+    assert np.abs(y - want).max() < 2e-6 * np.abs(want).max()        # fp32 butterfly vs float64 matmul
+    assert np.allclose((y ** 2).sum(1), (x.astype(np.float64) ** 2).sum(1), rtol=1e-5)   # norms preserved
+    # scores are invariant: (Q R)(K R)^T = Q K^T
+    k = rng.standard_normal((50, 128)).astype(np.float32)
+    s0 = x.astype(np.float64) @ k.astype(np.float64).T
+    s1 = y @ mxfp4.hadamard_rotate_f32(k).astype(np.float64).T
+    assert np.abs(s0 - s1).max() < 1e-4
+    # a one-hot row picks out a row of H / sqrt(n) exactly (up to the single fp32 scaling)
+    e = np.zeros((1, 128), np.float32); e[0, 37] = 1.0
+    assert np.array_equal(mxfp4.hadamard_rotate_f32(e)[0], (mxfp4.hadamard_matrix(128)[37] * np.float32(1 / np.sqrt(128.0))).astype(np.float32))
+
+
+def test_rotation_spreads_channel_outliers():
+    # the reason the rotation is there (Section 4.3): after it no channel dominates the block maxima
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((2000, 128)).astype(np.float32); x[:, [3, 40, 77]] *= 16
+    err = lambda z: float(((mxfp4.quantize_dequantize(z, 1, mxfp4.UOS) - z.astype(np.float64)) ** 2).sum() / (z.astype(np.float64) ** 2).sum())
+    assert err(mxfp4.hadamard_rotate_f32(x)) < err(x)

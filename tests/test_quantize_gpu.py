@@ -138,3 +138,37 @@ def test_power_of_two_scaling_shifts_scale_bytes_only():
     c0, s0 = run_gpu(bits, 512, 128, 1, 1)
     c1, s1 = run_gpu(si.f32_to_bf16_bits(x * np.float32(2.0 ** 9)), 512, 128, 1, 1)
     assert np.array_equal(c0, c1) and np.array_equal(s0.astype(np.int32) + 9, s1.astype(np.int32))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("rows", [1, 100, 1024, 4099])
+def test_hadamard_rotated_quantization_matches_oracle_bit_exact(rows, mode):
+    # Algorithm 2 lines 1-4: rotate, then quantize; fp32 butterfly order is part of the definition
+    import paper_2607_24377_b200 as mx
+    bits = gaussian_bits(rows, 128, 300 + rows + mode)
+    bits[::5, 7] = si.f32_to_bf16_bits(np.full(len(bits[::5]), 37.5, np.float32))      # a channel outlier
+    x = si.bf16_bits_to_f32(bits)
+    want_c, want_s = mxfp4.quantize_matrix_canonical(mxfp4.hadamard_rotate_f32(x).astype(np.float64), 1, RULE[mode])
+    codes = torch.zeros((rows, 64), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((rows, 4), dtype=torch.uint8, device="cuda")
+    mx.quantize_mxfp4_batched(util.to_dev_bf16(bits), codes, scales, 1, rows, 128, 1, mode | mx.MODE_HADAMARD, mx.LAYOUT_CANONICAL)
+    torch.cuda.synchronize()
+    assert np.array_equal(scales.cpu().numpy(), want_s)
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+    # tile layout: same values, permuted
+    nt = -(-rows // 128)
+    tc = torch.zeros((1, nt, 8192), dtype=torch.uint8, device="cuda"); ts = torch.zeros((1, nt, 512), dtype=torch.uint8, device="cuda")
+    mx.quantize_mxfp4_batched(util.to_dev_bf16(bits), tc, ts, 1, rows, 128, 1, mode | mx.MODE_HADAMARD, mx.LAYOUT_TILE)
+    torch.cuda.synchronize()
+    wc, ws = util.canonical_to_tile_axis1(want_c, want_s)
+    assert np.array_equal(ts[0].cpu().numpy(), ws) and np.array_equal(tc[0].cpu().numpy(), wc)
+
+
+def test_rotation_is_refused_where_it_is_not_defined():
+    import paper_2607_24377_b200 as mx
+    x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(128 * 256, dtype=torch.uint8, device="cuda")
+    for axis, cols in ((1, 256), (0, 128)):
+        with pytest.raises(mx.MxAttnError) as ei:
+            mx.quantize_mxfp4_batched(x, out, out, 1, 128, cols, axis, mx.MODE_UOS | mx.MODE_HADAMARD, mx.LAYOUT_CANONICAL)
+        assert ei.value.code == -2
