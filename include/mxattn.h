@@ -103,6 +103,15 @@ int mxattn_quantize_mxfp4_batched(const void* in, void* codes, void* e8m0_scales
                                   int64_t rows, int64_t cols, int block_axis, int mode, int layout,
                                   void* stream);
 
+/* The ceiling family with an arbitrary boundary: e = ceil(log2(M / qmax)) (paper Eq. 7), for the
+ * scale-rule comparisons of the paper: qmax = 6 is Truncation-Free Scaling (Eq. 8), 7 is the OAS rule at
+ * block size 32 (Appendix G), 7.25 is UOS, and a sweep over [6, 8] reproduces the setting of the
+ * paper's Q_max study (Section 5.4.1).  4 <= qmax < 16.  Other arguments as
+ * mxattn_quantize_mxfp4_batched. */
+int mxattn_quantize_mxfp4_qmax(const void* in, void* codes, void* e8m0_scales, int64_t batch,
+                               int64_t rows, int64_t cols, int block_axis, float qmax, int layout,
+                               void* stream);
+
 /* Bytes of device scratch the forward pass needs for the quantized Q, K, V tile images, their
  * scales and a status word.  0 if the shape is unsupported. */
 size_t mxattn_forward_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);

@@ -42,6 +42,7 @@ def lib() -> ctypes.CDLL:
                                    ctypes.c_uint, ctypes.c_size_t)
         L.mxattn_quantize_mxfp4.argtypes = [vp, vp, vp, i64, i64, ci, ci, vp]
         L.mxattn_quantize_mxfp4_batched.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, ci, vp]
+        L.mxattn_quantize_mxfp4_qmax.argtypes = [vp, vp, vp, i64, i64, i64, ci, cf, ci, vp]
         L.mxattn_forward_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_workspace_bytes.restype = sz
         L.mxattn_set_workspace.argtypes = [vp, sz]
@@ -86,6 +87,11 @@ def quantize_mxfp4_batched(inp, codes, e8m0_scales, batch, rows, cols, block_axi
     _check(lib().mxattn_quantize_mxfp4_batched(_ptr(inp), _ptr(codes), _ptr(e8m0_scales), batch, rows,
                                                cols, block_axis, mode, layout, _stream()),
            "mxattn_quantize_mxfp4_batched")
+
+
+def quantize_mxfp4_qmax(inp, codes, e8m0_scales, batch, rows, cols, block_axis, qmax, layout):
+    _check(lib().mxattn_quantize_mxfp4_qmax(_ptr(inp), _ptr(codes), _ptr(e8m0_scales), batch, rows, cols,
+                                            block_axis, qmax, layout, _stream()), "mxattn_quantize_mxfp4_qmax")
 
 
 def forward_workspace_bytes(B, H, Nq, Nkv, d) -> int:

@@ -28,6 +28,25 @@ __device__ __forceinline__ int shared_exponent(uint32_t u, bool uos) {
   return e < -127 ? -127 : e;
 }
 
+// The ceiling family e = ceil(log2(M / q)) for an arbitrary boundary q > 0 (paper Eq. 7; TFS is q = 6,
+// OAS at block 32 is q = 7, UOS is q = 7.25): with M = mu * 2^E and q = mu_q * 2^Eq,
+// e = E - Eq + [mu > mu_q], decided on the bit patterns.  `q_bits` is the fp32 pattern of q.
+__device__ __forceinline__ int shared_exponent_ceil(uint32_t u, uint32_t q_bits) {
+  if (u == 0u) return 0;
+  const int eb = (int)(u >> 23);
+  if (eb == 0) return -127;
+  const int e = eb - (int)(q_bits >> 23) + (((u & 0x7FFFFFu) > (q_bits & 0x7FFFFFu)) ? 1 : 0);
+  return e < -127 ? -127 : (e > 127 ? 127 : e);
+}
+
+// Rule word used by the quantize kernels: 0 = OCP floor rule, otherwise the fp32 bit pattern of the
+// ceiling-family boundary q (UOS: 7.25f).  For q = 7.25 this is exactly shared_exponent(u, true).
+constexpr uint32_t kRuleOcp = 0u;
+constexpr uint32_t kRuleUos = 0x40E80000u;   // 7.25f
+__device__ __forceinline__ int shared_exponent_rule(uint32_t u, uint32_t rule) {
+  return rule == kRuleOcp ? shared_exponent(u, false) : shared_exponent_ceil(u, rule);
+}
+
 // 2^-e as fp32 for e in [-127, 126] (exact, normal number).
 __device__ __forceinline__ float pow2_neg(int e) {
   return __uint_as_float((uint32_t)(127 - e) << 23);
@@ -70,7 +89,8 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // Internal launchers (defined in quantize.cu / forward.cu); all return an mxattn_status.
 int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, int64_t rows,
-                    int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream);
+                    int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream,
+                    uint32_t rule_override = 0xFFFFFFFFu);
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes,
                    const void* k_scales, const void* v_codes, const void* v_scales, void* o,
                    int B, int H, int64_t Nq, int64_t Nkv, float softmax_scale, unsigned flags,

@@ -7,6 +7,8 @@
 //     128-token x 128-column slab in shared memory with coalesced 128-bit loads, quantizes down
 //     the columns, and writes the transposed codes through a shared-memory staging tile so that
 //     the global stores stay 128-bit.
+#include <string.h>
+
 #include "common.cuh"
 
 namespace mxattn {
@@ -61,7 +63,7 @@ __device__ __forceinline__ void hadamard128_rows(float (&f)[8], int lane) {
 // 32-element block combine their maxima with two shuffles.  With kRotate the 16 lanes of a row
 // first apply the Hadamard rotation and the block maximum is taken on the fp32 results.
 template <bool kRotate>
-__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, bool uos, int* e_out) {
+__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, uint32_t rule, int* e_out) {
   if (kRotate) {
     float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y), bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
     hadamard128_rows(f, lane);
@@ -70,7 +72,7 @@ __device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, boo
     for (int i = 0; i < 8; ++i) m = max(m, __float_as_uint(f[i]) & 0x7FFFFFFFu);
     m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
     m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-    const int e = shared_exponent(m, uos);
+    const int e = shared_exponent_rule(m, rule);
     const float inv = pow2_neg(e);
     *e_out = e;
     return pack_e2m1x8(f[0] * inv, f[1] * inv, f[2] * inv, f[3] * inv, f[4] * inv, f[5] * inv, f[6] * inv, f[7] * inv);
@@ -78,7 +80,7 @@ __device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, boo
     uint32_t m = absmax_bf16x8(v);
     m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
     m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-    const int e = shared_exponent(m << 16, uos);
+    const int e = shared_exponent_rule(m << 16, rule);
     *e_out = e;
     return quantize_bf16x8(v, pow2_neg(e));
   }
@@ -93,7 +95,7 @@ constexpr int kQUnroll = 4;
 template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
-                      uint8_t* __restrict__ scales, int64_t n_chunks, bool uos) {
+                      uint8_t* __restrict__ scales, int64_t n_chunks, uint32_t rule) {
   const int lane = threadIdx.x & 31;
   const int64_t stride = (int64_t)gridDim.x * kQThreads;
   // warp-uniform loop bound: every lane of a warp runs the same number of iterations
@@ -109,7 +111,7 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
     for (int u = 0; u < kQUnroll; ++u) {
       const int64_t i = base + (int64_t)u * stride + lane;
       int e;
-      const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, uos, &e);
+      const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, rule, &e);
       // four consecutive blocks (16 lanes) -> one 32-bit scale word
       const uint32_t eb = (uint32_t)(e + 127);
       const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
@@ -139,7 +141,7 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
 template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
-                           uint8_t* __restrict__ scales, int64_t rows, bool uos) {
+                           uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t tile = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
   const int64_t row0 = (int64_t)blockIdx.x * kTile;
@@ -158,7 +160,7 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
     const int chunk = k * kQThreads + tid;
     const int r = chunk >> 4, c = (chunk >> 2) & 3;
     int e;
-    const uint32_t packed = quantize_chunk<kRotate>(v[k], lane, uos, &e);
+    const uint32_t packed = quantize_chunk<kRotate>(v[k], lane, rule, &e);
     const uint32_t eb = (uint32_t)(e + 127);
     const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
     const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
@@ -177,7 +179,7 @@ template <bool kTileLayout>
 __global__ void __launch_bounds__(kVThreads)
 quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t rows, int64_t cols, int64_t rows_pad,
-                      bool uos) {
+                      uint32_t rule) {
   __shared__ __align__(16) uint16_t s_in[kTile][kTile];           // [token][column] raw bf16
   __shared__ __align__(16) uint8_t s_codes[kTileCodeBytes];       // [column][64 B] (swizzled if tile layout)
   __shared__ __align__(16) uint8_t s_scales[kTileScaleBytes];
@@ -214,7 +216,7 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
       m = __vmaxu2(m, w[i] & 0x7FFF7FFFu);
     }
     m = max(m & 0xFFFFu, m >> 16);
-    const int e = shared_exponent(m << 16, uos);
+    const int e = shared_exponent_rule(m << 16, rule);
     const float inv = pow2_neg(e);
     uint4 out;
     out.x = pack_e2m1x8(bf16lo(w[0]) * inv, bf16hi(w[0]) * inv, bf16lo(w[1]) * inv, bf16hi(w[1]) * inv,
@@ -261,7 +263,8 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
 
 // ------------------------------------------------------------------------------------------
 int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, int64_t rows,
-                    int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream) {
+                    int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream,
+                    uint32_t rule_override) {
   if (!in || !codes || !scales) return MXATTN_EINVAL;
   if (batch <= 0 || rows <= 0 || cols <= 0) return MXATTN_EINVAL;
   if (block_axis != 0 && block_axis != 1) return MXATTN_EINVAL;
@@ -274,7 +277,7 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
   if (block_axis == 1 && cols % kBlock != 0) return MXATTN_EUNSUPPORTED;
   if (block_axis == 0 && cols % 8 != 0) return MXATTN_EUNSUPPORTED;
   if (!aligned16(in) || !aligned16(codes) || !aligned16(scales)) return MXATTN_EALIGN;
-  const bool uos = (mode == MXATTN_MODE_UOS);
+  const uint32_t rule = rule_override != 0xFFFFFFFFu ? rule_override : (mode == MXATTN_MODE_UOS ? kRuleUos : kRuleOcp);
   const int64_t rows_pad = (rows + kTile - 1) / kTile * kTile;
 
   if (block_axis == 1) {
@@ -289,17 +292,17 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
       if (rotate)
         quantize_axis1_tile_kernel<true><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
-                                                                         (uint8_t*)scales, rows, uos);
+                                                                         (uint8_t*)scales, rows, rule);
       else
         quantize_axis1_tile_kernel<false><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
-                                                                          (uint8_t*)scales, rows, uos);
+                                                                          (uint8_t*)scales, rows, rule);
     } else {
       if (rotate)
         quantize_axis1_kernel<true><<<(unsigned)blocks, kQThreads, 0, stream>>>(
-            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
+            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
       else
         quantize_axis1_kernel<false><<<(unsigned)blocks, kQThreads, 0, stream>>>(
-            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, uos);
+            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
     }
   } else {
     const int64_t ct = (cols + kTile - 1) / kTile, rt = rows_pad / kTile;
@@ -307,10 +310,10 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
     dim3 grid((unsigned)ct, (unsigned)rt, (unsigned)batch);
     if (layout == MXATTN_LAYOUT_TILE)
       quantize_axis0_kernel<true><<<grid, kVThreads, 0, stream>>>(
-          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, uos);
+          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, rule);
     else
       quantize_axis0_kernel<false><<<grid, kVThreads, 0, stream>>>(
-          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, uos);
+          (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, rule);
   }
   count_launch(1);
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
@@ -329,4 +332,14 @@ extern "C" int mxattn_quantize_mxfp4_batched(const void* in, void* codes, void* 
                                              int block_axis, int mode, int layout, void* stream) {
   return mxattn::launch_quantize(in, codes, e8m0_scales, batch, rows, cols, block_axis, mode, layout,
                                  (cudaStream_t)stream);
+}
+
+extern "C" int mxattn_quantize_mxfp4_qmax(const void* in, void* codes, void* e8m0_scales, int64_t batch,
+                                          int64_t rows, int64_t cols, int block_axis, float qmax,
+                                          int layout, void* stream) {
+  if (!(qmax >= 4.0f) || !(qmax < 16.0f)) return MXATTN_EINVAL;
+  uint32_t bits;
+  memcpy(&bits, &qmax, sizeof bits);
+  return mxattn::launch_quantize(in, codes, e8m0_scales, batch, rows, cols, block_axis, MXATTN_MODE_UOS, layout,
+                                 (cudaStream_t)stream, bits);
 }

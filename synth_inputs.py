@@ -71,6 +71,10 @@ CONFIGS = {
 for _n in (4096, 16384, 32768, 65536):  # BASELINE configs[4], the sweep
     CONFIGS[f"sweep{_n}"] = AttnConfig(f"sweep{_n}", 1, 40, _n, _n, 100 + int(math.log2(_n)), "outlier")
 
+# Wan2.2 has separate cross-attention modules (paper Section 5.1): video queries against a short text
+# context.  512 context tokens stand in for the text encoder's sequence.
+CONFIGS["wan22_cross"] = AttnConfig("wan22_cross", 1, 40, 75600, 512, 4, "wan")
+
 HUNYUAN_VIDEO_TOKENS = 118800
 
 

@@ -172,3 +172,42 @@ def test_rotation_is_refused_where_it_is_not_defined():
         with pytest.raises(mx.MxAttnError) as ei:
             mx.quantize_mxfp4_batched(x, out, out, 1, 128, cols, axis, mx.MODE_UOS | mx.MODE_HADAMARD, mx.LAYOUT_CANONICAL)
         assert ei.value.code == -2
+
+
+@pytest.mark.parametrize("qmax", [6.0, 7.0, 7.25, 6.55, 8.0, 4.0, 15.5])
+def test_generic_ceiling_boundary_matches_oracle(qmax):
+    # Eq. 7: the ceiling family; TFS (6), OAS at block 32 (7), UOS (7.25)
+    import paper_2607_24377_b200 as mx
+    rows = 777
+    bits = gaussian_bits(rows, 128, 400 + int(qmax * 100))
+    bits[0, :32] = si.f32_to_bf16_bits(np.full(32, qmax, np.float32))           # the endpoint q maps to exactly q
+    rule = mxfp4.ScaleRule("ceil", float(np.float32(qmax)))
+    for axis in (1, 0):
+        want_c, want_s = mxfp4.quantize_matrix_canonical(util.bits_to_f64(bits), axis, rule)
+        codes = torch.zeros(want_c.shape, dtype=torch.uint8, device="cuda")
+        scales = torch.zeros(want_s.shape, dtype=torch.uint8, device="cuda")
+        mx.quantize_mxfp4_qmax(util.to_dev_bf16(bits), codes, scales, 1, rows, 128, axis, qmax, mx.LAYOUT_CANONICAL)
+        torch.cuda.synchronize()
+        assert np.array_equal(scales.cpu().numpy(), want_s)
+        assert np.array_equal(codes.cpu().numpy(), want_c)
+
+
+def test_qmax_sweep_of_tensor_error_bottoms_near_7_25():
+    # the setting of the paper's Q_max study (Section 5.4.1) on a synthetic N(0,1) tensor: sweep 6.00 .. 8.00
+    import paper_2607_24377_b200 as mx
+    rows = 8192
+    bits = gaussian_bits(rows, 128, 500, spread=False)
+    x = util.bits_to_f64(bits)
+    dev = util.to_dev_bf16(bits)
+    codes = torch.zeros((rows, 64), dtype=torch.uint8, device="cuda"); scales = torch.zeros((rows, 4), dtype=torch.uint8, device="cuda")
+    mse = {}
+    for q in np.round(np.arange(6.0, 8.0001, 0.25), 2):
+        mx.quantize_mxfp4_qmax(dev, codes, scales, 1, rows, 128, 1, float(q), mx.LAYOUT_CANONICAL)
+        torch.cuda.synchronize()
+        c = codes.cpu().numpy(); s = scales.cpu().numpy().astype(np.int32) - 127
+        nib = np.stack([c & 15, c >> 4], axis=-1).reshape(rows, 4, 32)
+        deq = mxfp4.dequantize_blocks(nib, s).reshape(rows, 128)
+        mse[float(q)] = float(((deq - x) ** 2).mean())
+    best = min(mse, key=mse.get)
+    assert best in (7.0, 7.25, 7.5), mse
+    assert mse[7.25] < mse[6.0] and mse[7.25] < mse[8.0]
