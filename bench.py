@@ -278,9 +278,22 @@ def main():
         variants["quantize_q_with_hadamard"] = {"ms": ms, "GBps": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9,
                                                 "frac_of_hbm_peak": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, mx.MODE_UOS, mx.LAYOUT_TILE)       # restore the unrotated Q-hat
+        # bf16 variant of this repository's own kernel (no quantization; three re-tiling launches + attention)
+        wsb = torch.empty(mx.forward_bf16_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+        mx.forward_bf16(dq, dk, dv, out, B, H, Nq, Nkv, d, scale, 0, wsb); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(3):
+            mx.forward_bf16(dq, dk, dv, out, B, H, Nq, Nkv, d, scale, 0, wsb)
+        b.record(); torch.cuda.synchronize()
+        assert mx.device_status(wsb) == 0
+        ms = a.elapsed_time(b) / 3
+        variants["bf16_same_kernel"] = {"step_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                                        "note": "mxattn_forward_bf16: whole call (re-tiling of Q, K, V^T + fused attention)"}
+        variants["uos_pnq_step_speedup_over_bf16_same_kernel"] = ms / ms_per_step
+        del wsb
         # bf16 reference point: NOT a kernel of this repository -- PyTorch's fused SDPA (library flash /
-        # cuDNN attention) on the same bf16 tensors.  A bf16 (kind::f16) variant of this repo's own
-        # kernel is not built yet.
+        # cuDNN attention) on the same bf16 tensors.  (The repository's own bf16 variant is `bf16_same_kernel` above.)
         try:
             import torch.nn.functional as F
             ob = F.scaled_dot_product_attention(dq, dk, dv, scale=scale); del ob

@@ -147,6 +147,19 @@ int mxattn_forward_prequantized(const void* q_codes, const void* q_scales,
                                 int B, int H, int64_t Nq, int64_t Nkv, int d,
                                 float softmax_scale, unsigned flags, void* status, void* stream);
 
+/* bf16 variant of the same fused kernel, with no quantization anywhere: the FlashAttention-2
+ * recurrence the paper starts from (Section 2, Eq. 2-3) with bf16 operands on the tensor cores, the
+ * exponentials rounded to bf16 for the second GEMM and the row sum taken from the fp32 exponentials.
+ * It is the high-precision reference point for the MXFP4 variants (the paper's "FP16" baseline,
+ * Section 5.2).  Same tensor layouts as mxattn_forward; flags: only MXATTN_FLAG_OUT_FP32.
+ * The workspace holds re-tiled copies of Q, K and V^T (mxattn_forward_bf16_workspace_bytes, about the
+ * size of the inputs) and the status word at its start. */
+size_t mxattn_forward_bf16_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);
+int mxattn_forward_bf16(const void* q, const void* k, const void* v, void* o,
+                        int B, int H, int64_t Nq, int64_t Nkv, int d,
+                        float softmax_scale, unsigned flags,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of device memory mxattn_forward_host needs (inputs, output and workspace). */
 size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags);
 

@@ -129,3 +129,34 @@ def dense_attention_head(q, k, v, softmax_scale: float, rows=None) -> np.ndarray
     p = np.exp(s)
     p /= p.sum(axis=1, keepdims=True)
     return p @ v
+
+
+def _round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 round-to-nearest-even, returned as float64 (finite inputs)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
+def forward_head_bf16(q, k, v, softmax_scale: float, rows=None):
+    """The unquantized bf16 variant of the same recurrence (Section 2, Eq. 2-3; tiles of 128 keys):
+    bf16 Q, K, V as given, the exponentials rounded to bf16 (RNE) for the P V product, the row sum
+    taken from the fp32 exponentials."""
+    q = np.asarray(q, dtype=np.float64)
+    if rows is not None:
+        q = q[np.asarray(rows)]
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    nq, d = q.shape
+    scale = float(np.float32(softmax_scale))
+    m = np.full(nq, -np.inf); l = np.zeros(nq); o = np.zeros((nq, d))
+    for j0 in range(0, k.shape[0], B_C):
+        s = (q @ k[j0:j0 + B_C].T) * scale
+        m_new = np.maximum(m, s.max(axis=1))
+        alpha = np.exp(m - m_new)
+        with np.errstate(under="ignore"):
+            p32 = np.exp(s - m_new[:, None]).astype(np.float32)
+        l = alpha * l + p32.astype(np.float64).sum(axis=1)
+        o = alpha[:, None] * o + _round_to_bf16(p32) @ v[j0:j0 + B_C]
+        m = m_new
+    return o / l[:, None]

@@ -132,3 +132,23 @@ def test_full_algorithm_with_hadamard_rotation(recipe):
         e_rot = np.linalg.norm(got.double().cpu().numpy() - dense) / np.linalg.norm(dense)
         e_plain = np.linalg.norm(plain - dense) / np.linalg.norm(dense)
         assert e_rot < e_plain
+
+
+@pytest.mark.parametrize("nq,nkv", [(1024, 1024), (300, 1000), (77, 40), (640, 1296)])
+def test_bf16_variant_of_the_kernel(nq, nkv):
+    # the unquantized reference point: same recurrence, bf16 operands, P rounded to bf16, l from fp32 P
+    import paper_2607_24377_b200 as mx
+    cfg = si.custom_config("bf", 1, 2, nq, nkv, 300 + nq)
+    q, k, v = si.make_all(cfg)
+    out = torch.full((1, 2, nq, 128), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(mx.forward_bf16_workspace_bytes(1, 2, nq, nkv, 128), dtype=torch.uint8, device="cuda")
+    mx.forward_bf16(util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v), out, 1, 2, nq, nkv, 128,
+                    cfg.softmax_scale, mx.FLAG_OUT_FP32, ws)
+    assert mx.device_status(ws) == 0
+    f = util.bits_to_f64
+    want = np.stack([attention.forward_head_bf16(f(q[0, h]), f(k[0, h]), f(v[0, h]), cfg.softmax_scale) for h in range(2)])[None]
+    check(out, want)
+    # and it is close to float64 dense attention (bf16 rounding of P only)
+    dense = np.stack([attention.dense_attention_head(f(q[0, h]), f(k[0, h]), f(v[0, h]), cfg.softmax_scale) for h in range(2)])[None]
+    got = out.double().cpu().numpy()
+    assert np.linalg.norm(got - dense) / np.linalg.norm(dense) < 5e-3

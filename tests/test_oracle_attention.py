@@ -233,3 +233,13 @@ def test_rotation_with_identity_quantizer_changes_nothing():
     a = attention.forward_head(rq, rk, v, SCALE, quantize_inputs=False, quantize_p=False)
     b = attention.dense_attention_head(q, k, v, SCALE)
     assert np.abs(a - b).max() < 1e-5
+
+
+def test_bf16_variant_oracle_is_dense_attention_up_to_bf16_rounding_of_p():
+    q, k, v = head(64, 700, 25)
+    a = attention.forward_head_bf16(q, k, v, SCALE)
+    b = attention.dense_attention_head(q, k, v, SCALE)
+    assert 1e-6 < rel_l2(a, b) < 5e-3          # only P is rounded (2^-9 relative), and it must be rounded
+    # rounding helper: exact on bf16-representable values, RNE on a tie
+    r = attention._round_to_bf16(np.array([1.0, 1.00390625, 1.01171875, -3.0], np.float32))
+    assert list(r) == [1.0, 1.0, 1.015625, -3.0]
