@@ -1,6 +1,8 @@
 // C-ABI entry points that orchestrate the kernels: workspace carving, the three quantize
 // launches plus the fused attention launch (paper Algorithm 2, lines 3-19), and the host-buffer
 // end-to-end form.
+#include <vector>
+
 #include "common.cuh"
 
 namespace mxattn {
@@ -110,13 +112,38 @@ extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_sc
                         softmax_scale, flags, static_cast<int*>(status), (cudaStream_t)stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Host-buffer form.  Heads are independent, so the call is pipelined head by head over three
+// streams: host->device copies of head h+1 and the device->host copy of head h-1 overlap the
+// kernels of head h (PCIe is full duplex).  The two helper streams and the events are created on
+// first use, once per device, and kept for the life of the process; no device memory is allocated.
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  std::vector<cudaEvent_t> ev;
+};
+static HostPipe g_pipe[64];
+
+static HostPipe* host_pipe(size_t n_events) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe& hp = g_pipe[dev];
+  if (!hp.in && cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (!hp.out && cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  while (hp.ev.size() < n_events) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    hp.ev.push_back(e);
+  }
+  return &hp;
+}
+
 extern "C" size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags) {
   WorkspaceLayout w;
-  if (!carve(B, H, Nq, Nkv, d, &w)) return 0;
+  if (!carve(1, 1, Nq, Nkv, d, &w) || B <= 0 || H <= 0) return 0;     // one workspace slice per head
   const size_t bh = (size_t)B * H;
   const size_t qb = align_up(bh * (size_t)Nq * d * 2, 256), kb = align_up(bh * (size_t)Nkv * d * 2, 256);
   const size_t ob = align_up(bh * (size_t)Nq * d * ((flags & MXATTN_FLAG_OUT_FP32) ? 4 : 2), 256);
-  return qb + 2 * kb + ob + w.total;
+  return qb + 2 * kb + ob + bh * w.total;
 }
 
 extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
@@ -129,25 +156,54 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   if (!aligned16(device_arena)) return MXATTN_EALIGN;
   cudaStream_t stream = (cudaStream_t)stream_;
   const size_t bh = (size_t)B * H;
-  const size_t qn = bh * (size_t)Nq * d * 2, kn = bh * (size_t)Nkv * d * 2;
-  const size_t on = bh * (size_t)Nq * d * ((flags & MXATTN_FLAG_OUT_FP32) ? 4 : 2);
+  const size_t osz = (flags & MXATTN_FLAG_OUT_FP32) ? 4 : 2;
+  const size_t qh = (size_t)Nq * d * 2, kh = (size_t)Nkv * d * 2, oh = (size_t)Nq * d * osz;   // bytes per head
+  WorkspaceLayout w;
+  carve(1, 1, Nq, Nkv, d, &w);
   uint8_t* a = static_cast<uint8_t*>(device_arena);
   uint8_t* dq = a;
-  uint8_t* dk = dq + align_up(qn, 256);
-  uint8_t* dv = dk + align_up(kn, 256);
-  uint8_t* dout = dv + align_up(kn, 256);
-  uint8_t* ws = dout + align_up(on, 256);
-  if (cudaMemcpyAsync(dq, q_host, qn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
-  if (cudaMemcpyAsync(dk, k_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
-  if (cudaMemcpyAsync(dv, v_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return MXATTN_ECUDA;
-  const int rc = forward_ws(dq, dk, dv, dout, B, H, Nq, Nkv, d, softmax_scale, flags, ws,
-                            arena_bytes - (size_t)(ws - a), stream);
-  if (rc) return rc;
-  if (cudaMemcpyAsync(o_host, dout, on, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return MXATTN_ECUDA;
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return MXATTN_ECUDA;
-  int st = 0;
-  if (cudaMemcpy(&st, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
-  return st ? MXATTN_ETIMEOUT : MXATTN_OK;
+  uint8_t* dk = dq + align_up(bh * qh, 256);
+  uint8_t* dv = dk + align_up(bh * kh, 256);
+  uint8_t* dout = dv + align_up(bh * kh, 256);
+  uint8_t* ws = dout + align_up(bh * oh, 256);
+  HostPipe* hp = host_pipe(2 * bh + 2);
+  if (!hp) return MXATTN_ECUDA;
+  cudaEvent_t* ev = hp->ev.data();
+  bool fail = false;
+  auto ck = [&](cudaError_t e) { if (e != cudaSuccess) fail = true; };
+  ck(cudaEventRecord(ev[2 * bh], stream));                       // work already queued on the caller's stream comes first
+  ck(cudaStreamWaitEvent(hp->in, ev[2 * bh], 0));
+  int rc = MXATTN_OK;
+  for (size_t i = 0; i < bh && !fail && rc == MXATTN_OK; ++i) {
+    const char* qs = static_cast<const char*>(q_host) + i * qh;
+    const char* ks = static_cast<const char*>(k_host) + i * kh;
+    const char* vs = static_cast<const char*>(v_host) + i * kh;
+    ck(cudaMemcpyAsync(dq + i * qh, qs, qh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaMemcpyAsync(dk + i * kh, ks, kh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaMemcpyAsync(dv + i * kh, vs, kh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaEventRecord(ev[2 * i], hp->in));
+    ck(cudaStreamWaitEvent(stream, ev[2 * i], 0));
+    rc = forward_ws(dq + i * qh, dk + i * kh, dv + i * kh, dout + i * oh, 1, 1, Nq, Nkv, d, softmax_scale, flags,
+                    ws + i * w.total, w.total, stream);
+    ck(cudaEventRecord(ev[2 * i + 1], stream));
+    ck(cudaStreamWaitEvent(hp->out, ev[2 * i + 1], 0));
+    ck(cudaMemcpyAsync(static_cast<char*>(o_host) + i * oh, dout + i * oh, oh, cudaMemcpyDeviceToHost, hp->out));
+  }
+  ck(cudaEventRecord(ev[2 * bh + 1], hp->out));
+  ck(cudaStreamWaitEvent(stream, ev[2 * bh + 1], 0));
+  // everything enqueued so far must drain before returning, also on an error path
+  ck(cudaStreamSynchronize(hp->in));
+  ck(cudaStreamSynchronize(stream));
+  ck(cudaStreamSynchronize(hp->out));
+  g_launches = 4 * (int)bh;
+  if (rc != MXATTN_OK) return rc;
+  if (fail) return MXATTN_ECUDA;
+  // one status word per head, at the start of each workspace slice
+  std::vector<int> st(bh, 0);
+  if (cudaMemcpy2D(st.data(), sizeof(int), ws, w.total, sizeof(int), bh, cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  for (size_t i = 0; i < bh; ++i)
+    if (st[i]) return MXATTN_ETIMEOUT;
+  return MXATTN_OK;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -47,8 +47,14 @@
 namespace mxattn {
 namespace fwd {
 
-constexpr int kThreads = 576;                   // 16 softmax warps + producer + MMA issuer
-constexpr int kSoftmaxWarps = 16;
+#ifndef MXATTN_ROW_SPLIT
+#define MXATTN_ROW_SPLIT 2
+#endif
+constexpr int kSplit = MXATTN_ROW_SPLIT;         // threads per query row (1 or 2)
+constexpr int kCols = kTile / kSplit;            // key columns per softmax thread
+constexpr int kBlocksPerThread = 4 / kSplit;
+constexpr int kSoftmaxWarps = 8 * kSplit;
+constexpr int kThreads = 32 * (kSoftmaxWarps + 2);   // softmax warps + producer + MMA issuer
 constexpr int kStages = 4;
 constexpr int kNV = 144;                         // GEMM 2 N: 128 channels + 16 rows of ones
 constexpr int kVStageBytes = kNV * 64;           // 9216
@@ -127,8 +133,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
     }
     mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-    mbar_init(bar(BAR_SFREE), 8);                  // one arrival per softmax warp of the draining group
-    mbar_init(bar(BAR_PFULL + 0), 8); mbar_init(bar(BAR_PFULL + 1), 8);   // one arrival per softmax warp
+    mbar_init(bar(BAR_SFREE), 4 * kSplit);                  // one arrival per softmax warp of the draining group
+    mbar_init(bar(BAR_PFULL + 0), 4 * kSplit); mbar_init(bar(BAR_PFULL + 1), 4 * kSplit);   // one arrival per softmax warp
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -281,11 +287,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     }
   } else if (warp < kSoftmaxWarps) {
     // =============================== softmax groups =========================================
-    const int t = warp >> 3;                       // query tile of this group
-    const int h = (warp >> 2) & 1;                 // which 64 key columns of the tile
+    const int t = warp / (4 * kSplit);             // query tile of this group
+    const int h = kSplit == 2 ? ((warp >> 2) & 1) : 0;   // which key columns of the tile
     const int row = (warp & 3) * 32 + lane;        // row within the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_s = tmem + kColS + lane_addr + 64 * h;
+    const uint32_t t_s = tmem + kColS + lane_addr + kCols * h;
     const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;     // column 0 of this row's accumulator
     const float c = p.scale_log2e;
     float m_run = -INFINITY;
@@ -300,23 +306,23 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
       if (!ok) break;
       tc_fence_after();
-      uint32_t sr[64];
-      TMEM_LD32(t_s + 0, (sr + 0));
-      TMEM_LD32(t_s + 32, (sr + 32));
+      uint32_t sr[kCols];
+#pragma unroll
+      for (int c0 = 0; c0 < kCols; c0 += 32) TMEM_LD32(t_s + c0, (sr + c0));
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_SFREE));  // the score buffer may be overwritten
 
       if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
-        const int valid = (int)(p.Nkv - (int64_t)j * kTile) - 64 * h;
+        const int valid = (int)(p.Nkv - (int64_t)j * kTile) - kCols * h;
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
+        for (int i = 0; i < kCols; ++i)
           if (i >= valid) sr[i] = 0xFF800000u;     // -inf
       }
-      float bmax[2];
+      float bmax[kBlocksPerThread];
 #pragma unroll
-      for (int b = 0; b < 2; ++b) {                 // four independent chains of 8, then combine
+      for (int b = 0; b < kBlocksPerThread; ++b) {  // four independent chains of 8, then combine
         float q4[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -328,14 +334,22 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
         bmax[b] = fmaxf(max3(q4[0], q4[1], q4[2]), q4[3]);
       }
-      // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
-      float* mslot = sMax + ((j & 1) * 2 + t) * 256;
-      mslot[h * 128 + row] = fmaxf(bmax[0], bmax[1]);
+      float own_max = bmax[0];
+#pragma unroll
+      for (int b = 1; b < kBlocksPerThread; ++b) own_max = fmaxf(own_max, bmax[b]);
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t
-      // or rescales O_t; probe that barrier now so its latency overlaps the pair barrier
+      // or rescales O_t; probe that barrier early so its latency overlaps other work
       const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
-      const float m_new = max3(m_run, fmaxf(bmax[0], bmax[1]), mslot[(h ^ 1) * 128 + row]);        // line 10
+      float m_new;
+      if (kSplit == 2) {
+        // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
+        float* mslot = sMax + ((j & 1) * 2 + t) * 256;
+        mslot[h * 128 + row] = own_max;
+        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");    // only the two warps that share these rows
+        m_new = max3(m_run, own_max, mslot[(h ^ 1) * 128 + row]);      // line 10
+      } else {
+        m_new = fmaxf(m_run, own_max);                                 // line 10
+      }
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
@@ -359,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         constexpr bool kResc = decltype(resc_tag)::value;
         if (kResc) alpha = ex2((m_old - m_new) * c);
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kBlocksPerThread; ++b) {
           // Shared exponent of the block from d = log2(pmax) = (bmax_b - m_new) * c <= 0, with no
           // exponential: floor(log2 pmax) = floor(d), and the UOS rule raises the exponent iff the
           // mantissa 2^(d - floor d) exceeds 1.8125, i.e. iff frac(d) > log2(1.8125).  d = 0 (the
@@ -379,7 +393,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
 #pragma unroll
           for (int g = 0; g < 4; ++g) {             // 8 elements per step (8 accumulator columns in flight)
             uint32_t oc[8];
-            const uint32_t t_oc = t_o + 64 * h + 32 * b + 8 * g;
+            const uint32_t t_oc = t_o + kCols * h + 32 * b + 8 * g;
             if (kResc) TMEM_LD8(t_oc, oc);
             float x[8];
 #pragma unroll
@@ -394,7 +408,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
               TMEM_ST8(t_oc, oc);
             }
           }
-          *reinterpret_cast<uint4*>(sP + tile_code_offset(row, 2 * h + b)) = w;
+          *reinterpret_cast<uint4*>(sP + tile_code_offset(row, kBlocksPerThread * h + b)) = w;
           sf_half |= (uint32_t)(e + 127) << (8 * b);
           if (!kPnq) l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);   // Eq. 12
         }
@@ -410,7 +424,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       };
       if (rescale) tile_body(std::true_type{}); else tile_body(std::false_type{});
-      *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
+      if (kSplit == 2) *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
+      else *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_half;
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
@@ -421,7 +436,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     // ---- epilogue: O = O~ / l (line 18) ----
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
     float l = l_run;
-    if (!kPnq) {                                   // add the partner's half of the row sum
+    if (!kPnq && kSplit == 2) {                    // add the partner's half of the row sum
       float* mslot = sMax + ((T & 1) * 2 + t) * 256;
       mslot[h * 128 + row] = l_run;
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
@@ -438,11 +453,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         l = __uint_as_float(lr);
       }
       const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
-      const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + 64 * h;
+      const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + kCols * h;
 #pragma unroll 1
-      for (int c0 = 0; c0 < 64; c0 += 32) {
+      for (int c0 = 0; c0 < kCols; c0 += 32) {
         uint32_t r32[32];
-        TMEM_LD32(t_o + 64 * h + c0, r32);
+        TMEM_LD32(t_o + kCols * h + c0, r32);
         tmem_ld_wait();
         if (store) {
           if (kOutF32) {
