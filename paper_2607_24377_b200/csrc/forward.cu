@@ -367,27 +367,37 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       // lines 12-13: exponentials, already divided by the block scale, rounded to E2M1.  Two
       // straight-line versions: the common one, and one that also rescales this thread's 64
       // accumulator columns with the tensor-memory round trips interleaved into the exponentials.
+      // Shared exponent of each block from d = log2(pmax) = (bmax_b - m_new) * c <= 0, with no
+      // exponential: floor(log2 pmax) = floor(d), and the UOS rule raises the exponent iff the
+      // mantissa 2^(d - floor d) exceeds 1.8125, i.e. iff frac(d) > log2(1.8125).  d = 0 (the
+      // block holding the row maximum) gives e = -2 under both rules, as Appendix J derives.
+      // A block whose maximum underflows fp32 (d < -126, or fully masked) is a zero block.
+      float nbs[kBlocksPerThread], sigma[kBlocksPerThread];
       uint32_t sf_half = 0;
+#pragma unroll
+      for (int b = 0; b < kBlocksPerThread; ++b) {
+        const float d = (bmax[b] - m_new) * c;
+        const float rn = (d + 12582912.0f) - 12582912.0f;              // round to nearest integer
+        const float fl = rn > d ? rn - 1.0f : rn;                       // floor(d)
+        float ef = fl - 2.0f;
+        if (kUos && (d - fl) > 0.85798097f) ef += 1.0f;
+        ef = fmaxf(ef, -127.0f);
+        if (d < -126.0f) ef = 0.0f;
+        const int e = __float_as_int(ef + 12582912.0f) - 0x4B400000;    // exact small-integer conversion
+        nbs[b] = nmc - ef;
+        sigma[b] = __uint_as_float((uint32_t)(127 + e) << 23);          // 2^e (direct placement only)
+        sf_half |= (uint32_t)(e + 127) << (8 * b);
+      }
+      // the scale bytes go out before the exponentials, so only the code stores precede the proxy fence
+      if (kSplit == 2) *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
+      else *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_half;
       float l_tile = 0.0f;
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
         if (kResc) alpha = ex2((m_old - m_new) * c);
 #pragma unroll
         for (int b = 0; b < kBlocksPerThread; ++b) {
-          // Shared exponent of the block from d = log2(pmax) = (bmax_b - m_new) * c <= 0, with no
-          // exponential: floor(log2 pmax) = floor(d), and the UOS rule raises the exponent iff the
-          // mantissa 2^(d - floor d) exceeds 1.8125, i.e. iff frac(d) > log2(1.8125).  d = 0 (the
-          // block holding the row maximum) gives e = -2 under both rules, as Appendix J derives.
-          // A block whose maximum underflows fp32 (d < -126, or fully masked) is a zero block.
-          const float d = (bmax[b] - m_new) * c;
-          const float rn = (d + 12582912.0f) - 12582912.0f;            // round to nearest integer
-          const float fl = rn > d ? rn - 1.0f : rn;                     // floor(d)
-          float ef = fl - 2.0f;
-          if (kUos && (d - fl) > 0.85798097f) ef += 1.0f;
-          ef = fmaxf(ef, -127.0f);
-          if (d < -126.0f) ef = 0.0f;
-          const int e = __float_as_int(ef + 12582912.0f) - 0x4B400000;  // exact small-integer conversion
-          const float nb = nmc - ef;
+          const float nb = nbs[b];
           uint4 w;
           float sx = 0.0f;
 #pragma unroll
@@ -409,8 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
             }
           }
           *reinterpret_cast<uint4*>(sP + tile_code_offset(row, kBlocksPerThread * h + b)) = w;
-          sf_half |= (uint32_t)(e + 127) << (8 * b);
-          if (!kPnq) l_tile = fmaf(sx, __uint_as_float((uint32_t)(127 + e) << 23), l_tile);   // Eq. 12
+          if (!kPnq) l_tile = fmaf(sx, sigma[b], l_tile);   // Eq. 12
         }
         if (kResc) {
           if (kPnq && h == 0) {                     // column 128: the running row sum P-hat 1
@@ -424,8 +433,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         }
       };
       if (rescale) tile_body(std::true_type{}); else tile_body(std::false_type{});
-      if (kSplit == 2) *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
-      else *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_half;
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
