@@ -202,34 +202,36 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
   }
   __syncthreads();
 
-  // phase 2: thread -> (column n, token block c); 512 jobs, 2 per thread
+  // phase 2: thread -> (column pair 2np, 2np+1; token block c).  One 32-bit shared load brings both
+  // columns of a token, so the packed maximum and the two conversions share the 32 loads.
+  {
+    const int np = tid & 63, c = tid >> 6;
+    const uint32_t* s32 = reinterpret_cast<const uint32_t*>(&s_in[0][0]);
+    uint32_t w[32];
+    uint32_t m2 = 0;
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    const int n = tid & 127;
-    const int c = (tid >> 7) + 2 * k;
-    uint32_t w[16];
-    uint32_t m = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const uint32_t lo = s_in[c * 32 + 2 * i][n], hi = s_in[c * 32 + 2 * i + 1][n];
-      w[i] = lo | (hi << 16);
-      m = __vmaxu2(m, w[i] & 0x7FFF7FFFu);
+    for (int i = 0; i < 32; ++i) {
+      w[i] = s32[(c * 32 + i) * (kTile / 2) + np];
+      m2 = __vmaxu2(m2, w[i] & 0x7FFF7FFFu);
     }
-    m = max(m & 0xFFFFu, m >> 16);
-    const int e = shared_exponent_rule(m << 16, rule);
-    const float inv = pow2_neg(e);
-    uint4 out;
-    out.x = pack_e2m1x8(bf16lo(w[0]) * inv, bf16hi(w[0]) * inv, bf16lo(w[1]) * inv, bf16hi(w[1]) * inv,
-                        bf16lo(w[2]) * inv, bf16hi(w[2]) * inv, bf16lo(w[3]) * inv, bf16hi(w[3]) * inv);
-    out.y = pack_e2m1x8(bf16lo(w[4]) * inv, bf16hi(w[4]) * inv, bf16lo(w[5]) * inv, bf16hi(w[5]) * inv,
-                        bf16lo(w[6]) * inv, bf16hi(w[6]) * inv, bf16lo(w[7]) * inv, bf16hi(w[7]) * inv);
-    out.z = pack_e2m1x8(bf16lo(w[8]) * inv, bf16hi(w[8]) * inv, bf16lo(w[9]) * inv, bf16hi(w[9]) * inv,
-                        bf16lo(w[10]) * inv, bf16hi(w[10]) * inv, bf16lo(w[11]) * inv, bf16hi(w[11]) * inv);
-    out.w = pack_e2m1x8(bf16lo(w[12]) * inv, bf16hi(w[12]) * inv, bf16lo(w[13]) * inv, bf16hi(w[13]) * inv,
-                        bf16lo(w[14]) * inv, bf16hi(w[14]) * inv, bf16lo(w[15]) * inv, bf16hi(w[15]) * inv);
-    const int coff = kTileLayout ? tile_code_offset(n, c) : (n * 64 + c * 16);
-    *reinterpret_cast<uint4*>(&s_codes[coff]) = out;
-    s_scales[kTileLayout ? tile_scale_offset(n, c) : (n * 4 + c)] = (uint8_t)(e + 127);
+#pragma unroll
+    for (int side = 0; side < 2; ++side) {          // side 0: column 2np (low halves), side 1: column 2np+1
+      const int n = 2 * np + side;
+      const uint32_t m = side ? (m2 >> 16) : (m2 & 0xFFFFu);
+      const int e = shared_exponent_rule(m << 16, rule);
+      const float inv = pow2_neg(e);
+      uint32_t o[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = (side ? bf16hi(w[8 * q + i]) : bf16lo(w[8 * q + i])) * inv;
+        o[q] = pack_e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
+      }
+      const int coff = kTileLayout ? tile_code_offset(n, c) : (n * 64 + c * 16);
+      *reinterpret_cast<uint4*>(&s_codes[coff]) = make_uint4(o[0], o[1], o[2], o[3]);
+      s_scales[kTileLayout ? tile_scale_offset(n, c) : (n * 4 + c)] = (uint8_t)(e + 127);
+    }
   }
   __syncthreads();
 
