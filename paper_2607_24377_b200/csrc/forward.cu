@@ -307,8 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[kCols];
-#pragma unroll
-      for (int c0 = 0; c0 < kCols; c0 += 32) TMEM_LD32(t_s + c0, (sr + c0));
+      TMEM_LD64(t_s, sr);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
