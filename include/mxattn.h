@@ -215,6 +215,13 @@ int mxattn_forward_static(const void* q, const void* k, const void* v, void* o,
  * 0 = no bounded wait expired since the workspace was last used by a forward. */
 int mxattn_device_status(const void* workspace, int* host_out, void* stream);
 
+/* Exercises the failure path of the device-side waits without disturbing the GPU: a one-warp kernel
+ * waits on a barrier that nothing arrives on, gives up after `limit_cycles` SM cycles (at most 2e9) and
+ * writes the code 77 into status[0] (4 device ints, zeroed by the caller).  The kernel ends normally
+ * and the context stays usable.  Every wait inside the attention kernels uses the same routine with a
+ * limit of about two seconds. */
+int mxattn_selftest_bounded_wait(void* status, int64_t limit_cycles, void* stream);
+
 /* Number of kernel launches the last forward call of this process enqueued (for accounting). */
 int mxattn_last_launch_count(void);
 

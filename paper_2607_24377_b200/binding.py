@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_host_arena_bytes.restype = sz
         L.mxattn_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
         L.mxattn_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
+        L.mxattn_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.mxattn_last_launch_count.argtypes = []
         L.mxattn_strerror.argtypes = [ci]
         L.mxattn_strerror.restype = ctypes.c_char_p
@@ -163,6 +164,10 @@ def device_status(workspace) -> int:
     out = ctypes.c_int(0)
     _check(lib().mxattn_device_status(_ptr(workspace), ctypes.byref(out), _stream()), "mxattn_device_status")
     return out.value
+
+
+def selftest_bounded_wait(status, limit_cycles: int):
+    _check(lib().mxattn_selftest_bounded_wait(_ptr(status), int(limit_cycles), _stream()), "mxattn_selftest_bounded_wait")
 
 
 def last_launch_count() -> int:

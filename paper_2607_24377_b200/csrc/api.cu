@@ -266,6 +266,12 @@ extern "C" int mxattn_device_status(const void* workspace, int* host_out, void* 
   return MXATTN_OK;
 }
 
+extern "C" int mxattn_selftest_bounded_wait(void* status, int64_t limit_cycles, void* stream) {
+  if (!status || limit_cycles <= 0 || limit_cycles > 2000000000LL) return MXATTN_EINVAL;
+  if (!aligned16(status)) return MXATTN_EALIGN;
+  return launch_bounded_wait_selftest(static_cast<int*>(status), (long long)limit_cycles, (cudaStream_t)stream);
+}
+
 extern "C" int mxattn_last_launch_count(void) { return g_launches; }
 
 extern "C" const char* mxattn_strerror(int status) {

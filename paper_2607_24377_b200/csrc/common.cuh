@@ -98,6 +98,7 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
 size_t bf16_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv);
 int launch_forward_bf16(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq, int64_t Nkv,
                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream_t stream);
 void count_launch(int n);
 
 }  // namespace mxattn

@@ -499,7 +499,27 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever arrives on, with a
+// short limit; the wait must give up, record its code in `status`, and the kernel must end normally.
+__global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles) {
+  __shared__ uint64_t barrier;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&barrier), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool done = mbar_wait(smem_u32(&barrier), 0u, &abort_flag, status, 77, limit_cycles);
+  if (done && threadIdx.x == 0) atomicCAS(status, 0, -1);      // must not happen
+}
+
 }  // namespace fwd
+
+int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream_t stream) {
+  fwd::bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);
+  return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
+}
 
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes, const void* k_scales,
                    const void* v_codes, const void* v_scales, void* o, int B, int H, int64_t Nq, int64_t Nkv,

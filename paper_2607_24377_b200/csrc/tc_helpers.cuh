@@ -56,14 +56,14 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {     /
 // the CTA already gave up); the caller then skips to the teardown.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at full clock
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code) {
+                                          int* status, int code, long long limit = kWaitLimitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
     if ((it & 15) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;

@@ -152,3 +152,21 @@ def test_bf16_variant_of_the_kernel(nq, nkv):
     dense = np.stack([attention.dense_attention_head(f(q[0, h]), f(k[0, h]), f(v[0, h]), cfg.softmax_scale) for h in range(2)])[None]
     got = out.double().cpu().numpy()
     assert np.linalg.norm(got - dense) / np.linalg.norm(dense) < 5e-3
+
+
+def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
+    # failure detection without a fault: a wait that nothing satisfies runs out after a short limit,
+    # records its code, the kernel ends normally and the next forward on the same context is correct
+    import paper_2607_24377_b200 as mx
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    mx.selftest_bounded_wait(status, 2_000_000)          # about a millisecond of SM cycles
+    t1.record(); torch.cuda.synchronize()
+    assert int(status[0]) == 77
+    assert t0.elapsed_time(t1) < 200.0
+    cfg = si.custom_config("after", 1, 1, 130, 260, 5)
+    q, k, v = si.make_all(cfg)
+    check(run_forward(cfg, q, k, v, True, True), oracle_out(cfg, q, k, v, True, True))
+    with pytest.raises(mx.MxAttnError):
+        mx.selftest_bounded_wait(status, 0)
