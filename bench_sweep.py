@@ -1,0 +1,110 @@
+#!/usr/bin/env python
+"""Sweep report (BASELINE configs[1] and configs[4]); prints one JSON document.
+
+    python bench_sweep.py [--quick]
+
+* attention: N in {4096, 16384, 32768, 65536}, H=40, d=128, variants {bf16 (this repo's kernel),
+  OCP direct, UOS direct, UOS+PNQ, UOS+PNQ+Hadamard}: kernel-only ms / TFLOP/s, whole-step ms, and the
+  relative L2 error against float64 dense attention on sampled rows (CPU oracle);
+* outlier config (H=24, N=8192): the same quality comparison;
+* quantize: 2^20 .. 2^29 bf16 elements, axis 1 and axis 0, OCP and UOS: GB/s and fraction of the
+  measured HBM copy rate.
+
+The contract benchmark is bench.py; this script only adds the sweep tables.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+from bench import QUANT_BYTES_PER_ELEM, load_peaks  # noqa: E402
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true", help="smallest sizes only")
+    args = ap.parse_args()
+    import torch
+    import paper_2607_24377_b200 as mx
+    from oracle import attention
+    peaks = load_peaks()
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).cuda().view(torch.bfloat16)
+    f64 = lambda a: si.bf16_bits_to_f32(a).astype(np.float64)
+
+    def timed(fn, n=3):
+        fn(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    def attention_report(cfg, heads_for_quality=(0, 1), rows_per_head=32):
+        B, H, Nq, Nkv, d = cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d
+        q, k, v = si.make_all(cfg)
+        dq, dk, dv = dev(q), dev(k), dev(v)
+        out = torch.empty((B, H, Nq, d), dtype=torch.float32, device="cuda")
+        ws = torch.empty(mx.forward_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+        wsb = torch.empty(mx.forward_bf16_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+        rows = {h: np.sort(np.random.default_rng([5, h]).choice(Nq, rows_per_head, replace=False)) for h in heads_for_quality}
+        dense = {h: attention.dense_attention_head(f64(q[0, h]), f64(k[0, h]), f64(v[0, h]), cfg.softmax_scale, rows=rows[h])
+                 for h in heads_for_quality}
+
+        def quality():
+            num = den = 0.0
+            for h in heads_for_quality:
+                got = out[0, h][torch.from_numpy(rows[h]).cuda()].double().cpu().numpy()
+                num += float(((got - dense[h]) ** 2).sum()); den += float((dense[h] ** 2).sum())
+            return (num / den) ** 0.5
+
+        rep = {"B": B, "H": H, "N": Nq, "flops": cfg.flops, "variants": {}}
+        F32 = mx.FLAG_OUT_FP32
+        for name, fl in (("ocp_direct", 0), ("uos_direct", mx.FLAG_UOS), ("uos_pnq", mx.FLAG_UOS | mx.FLAG_PNQ),
+                         ("uos_pnq_hadamard", mx.FLAG_UOS | mx.FLAG_PNQ | mx.FLAG_HADAMARD)):
+            ms = timed(lambda: mx.forward_ws(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, fl | F32, ws))
+            assert mx.device_status(ws) == 0
+            rep["variants"][name] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
+        ms = timed(lambda: mx.forward_bf16(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, F32, wsb))
+        assert mx.device_status(wsb) == 0
+        rep["variants"]["bf16_same_kernel"] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
+        return rep
+
+    doc = {"peaks": peaks, "attention_sweep": [], "quantize_sweep": []}
+    sizes = (4096,) if args.quick else (4096, 16384, 32768, 65536)
+    for n in sizes:
+        doc["attention_sweep"].append(attention_report(si.CONFIGS[f"sweep{n}"]))
+        torch.cuda.empty_cache()
+    doc["outlier_config"] = attention_report(si.CONFIGS["outlier"], heads_for_quality=(0, 7, 15, 23), rows_per_head=16)
+    torch.cuda.empty_cache()
+
+    exps = (20, 24) if args.quick else range(20, 30)
+    for e in exps:
+        n = 1 << e
+        rows = n // 128
+        x = torch.randn((rows, 128), device="cuda").to(torch.bfloat16)
+        for axis in (1, 0):
+            batch = max(1, rows // 8192) if axis == 0 else 1
+            r = rows // batch
+            rp = -(-r // 128) * 128
+            codes = torch.empty(batch * max(r, rp) * 64 if axis == 1 else batch * 128 * rp // 2, dtype=torch.uint8, device="cuda")
+            scales = torch.empty(batch * max(r, rp) * 4, dtype=torch.uint8, device="cuda")
+            for mode, mname in ((mx.MODE_OCP, "ocp"), (mx.MODE_UOS, "uos")):
+                ms = timed(lambda: mx.quantize_mxfp4_batched(x, codes, scales, batch, r, 128, axis, mode, mx.LAYOUT_CANONICAL), n=10)
+                gbs = QUANT_BYTES_PER_ELEM * n / ms / 1e6
+                doc["quantize_sweep"].append({"elements": n, "axis": axis, "mode": mname, "ms": ms, "GBps": gbs,
+                                              "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
+        del x
+    print(json.dumps(doc))
+
+
+if __name__ == "__main__":
+    main()
