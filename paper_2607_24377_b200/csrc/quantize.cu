@@ -87,47 +87,45 @@ __device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, uin
 }
 
 constexpr int kQThreads = 256;
-constexpr int kQUnroll = 4;
 
 // ------------------------------------------------------------------------------------------
 // Axis 1, canonical layout: a linear streaming pass.  Work unit = one 16-byte chunk (8 elements);
-// chunk i yields code word i and (with its three neighbours) scale byte i / 4.
+// chunk i yields code word i and (with its three neighbours) scale byte i / 4.  A CTA owns 2048
+// consecutive chunks (32 KiB) and issues all of its loads before it quantizes anything.
+constexpr int kQChunksPerThread = 8;
+
 template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t n_chunks, uint32_t rule) {
   const int lane = threadIdx.x & 31;
-  const int64_t stride = (int64_t)gridDim.x * kQThreads;
-  // warp-uniform loop bound: every lane of a warp runs the same number of iterations
-  const int64_t warp_first = (int64_t)blockIdx.x * kQThreads + (threadIdx.x & ~31);
-  for (int64_t base = warp_first; base < n_chunks; base += stride * kQUnroll) {
-    uint4 v[kQUnroll];
+  const int64_t base = (int64_t)blockIdx.x * (kQThreads * kQChunksPerThread) + threadIdx.x;
+  uint4 v[kQChunksPerThread];
 #pragma unroll
-    for (int u = 0; u < kQUnroll; ++u) {
-      const int64_t i = base + (int64_t)u * stride + lane;
-      v[u] = i < n_chunks ? __ldg(in + i) : make_uint4(0u, 0u, 0u, 0u);
-    }
+  for (int u = 0; u < kQChunksPerThread; ++u) {
+    const int64_t i = base + u * kQThreads;
+    v[u] = i < n_chunks ? __ldg(in + i) : make_uint4(0u, 0u, 0u, 0u);
+  }
 #pragma unroll
-    for (int u = 0; u < kQUnroll; ++u) {
-      const int64_t i = base + (int64_t)u * stride + lane;
-      int e;
-      const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, rule, &e);
-      // four consecutive blocks (16 lanes) -> one 32-bit scale word
-      const uint32_t eb = (uint32_t)(e + 127);
-      const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
-      const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
-      const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
-      if (i >= n_chunks) continue;
-      codes[i] = packed;
-      if ((lane & 15) == 0) {
-        const int64_t g = i >> 2;                    // block index, multiple of 4 here
-        if (i + 16 <= n_chunks) {
-          *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
-        } else {                                     // ragged end: fewer than 4 blocks left
-          scales[g] = (uint8_t)eb;
-          if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
-          if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
-        }
+  for (int u = 0; u < kQChunksPerThread; ++u) {
+    const int64_t i = base + u * kQThreads;
+    int e;
+    const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, rule, &e);
+    // four consecutive blocks (16 lanes) -> one 32-bit scale word
+    const uint32_t eb = (uint32_t)(e + 127);
+    const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
+    const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
+    const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
+    if (i >= n_chunks) continue;
+    codes[i] = packed;
+    if ((lane & 15) == 0) {
+      const int64_t g = i >> 2;                      // block index, multiple of 4 here
+      if (i + 16 <= n_chunks) {
+        *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
+      } else {                                       // ragged end: fewer than 4 blocks left
+        scales[g] = (uint8_t)eb;
+        if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
+        if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
       }
     }
   }
@@ -285,10 +283,8 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
   if (block_axis == 1) {
     const bool tile = (layout == MXATTN_LAYOUT_TILE);
     const int64_t n_chunks = tile ? batch * rows_pad * 16 : batch * rows * (cols / 8);
-    int64_t blocks = (n_chunks + (int64_t)kQThreads * kQUnroll - 1) / ((int64_t)kQThreads * kQUnroll);
-    const int64_t cap = 148 * 8 * 4;                       // a few waves of resident CTAs
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
+    const int64_t blocks = (n_chunks + kQThreads * kQChunksPerThread - 1) / (kQThreads * kQChunksPerThread);
+    if (!tile && blocks > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
     if (tile) {
       if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
