@@ -47,10 +47,7 @@
 namespace mxattn {
 namespace fwd {
 
-#ifndef MXATTN_ROW_SPLIT
-#define MXATTN_ROW_SPLIT 2
-#endif
-constexpr int kSplit = MXATTN_ROW_SPLIT;         // threads per query row (1 or 2)
+constexpr int kSplit = 2;                        // threads per query row (one per row measured 25 % slower)
 constexpr int kCols = kTile / kSplit;            // key columns per softmax thread
 constexpr int kBlocksPerThread = 4 / kSplit;
 constexpr int kSoftmaxWarps = 8 * kSplit;
@@ -287,8 +284,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     }
   } else if (warp < kSoftmaxWarps) {
     // =============================== softmax groups =========================================
-    const int t = warp / (4 * kSplit);             // query tile of this group
-    const int h = kSplit == 2 ? ((warp >> 2) & 1) : 0;   // which key columns of the tile
+    const int t = warp >> 3;                       // query tile of this group
+    const int h = (warp >> 2) & 1;                 // which 64 key columns of the tile
     const int row = (warp & 3) * 32 + lane;        // row within the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t t_s = tmem + kColS + lane_addr + kCols * h;
@@ -296,9 +293,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     const float c = p.scale_log2e;
     float m_run = -INFINITY;
     float l_run = 0.0f;                            // direct placement only (this thread's 64 columns)
-    uint8_t* sP = smem + kOffP + t * kTileCodeBytes;
-    uint8_t* sSFP = smem + kOffSFP + t * kTileScaleBytes;
-    float* sMax = reinterpret_cast<float*>(smem + kOffMax);
+    // shared-space byte addresses of this thread's slots: its two 16-byte code chunks, its two scale
+    // bytes, and the half-row maximum exchange (own slot / partner's slot; + 2048 on odd tiles)
+    const uint32_t aP0 = sbase + kOffP + t * kTileCodeBytes + tile_code_offset(row, 2 * h);
+    const uint32_t aP1 = sbase + kOffP + t * kTileCodeBytes + tile_code_offset(row, 2 * h + 1);
+    const uint32_t aSF = sbase + kOffSFP + t * kTileScaleBytes + tile_scale_offset(row, 2 * h);
+    const uint32_t aMaxOwn = sbase + kOffMax + (t * 256 + h * 128 + row) * 4;
+    const uint32_t aMaxPartner = sbase + kOffMax + (t * 256 + (h ^ 1) * 128 + row) * 4;
     const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
     bool ok = true;
 
@@ -339,16 +340,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t
       // or rescales O_t; probe that barrier early so its latency overlaps other work
       const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
-      float m_new;
-      if (kSplit == 2) {
-        // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
-        float* mslot = sMax + ((j & 1) * 2 + t) * 256;
-        mslot[h * 128 + row] = own_max;
-        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");    // only the two warps that share these rows
-        m_new = max3(m_run, own_max, mslot[(h ^ 1) * 128 + row]);      // line 10
-      } else {
-        m_new = fmaxf(m_run, own_max);                                 // line 10
-      }
+      // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
+      const uint32_t par = (uint32_t)(j & 1) * 2048u;
+      sts32f(aMaxOwn + par, own_max);
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
+      const float m_new = max3(m_run, own_max, lds32f(aMaxPartner + par));   // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
@@ -388,8 +384,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         sf_half |= (uint32_t)(e + 127) << (8 * b);
       }
       // the scale bytes go out before the exponentials, so only the code stores precede the proxy fence
-      if (kSplit == 2) *reinterpret_cast<uint16_t*>(sSFP + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
-      else *reinterpret_cast<uint32_t*>(sSFP + tile_scale_offset(row, 0)) = sf_half;
+      sts16(aSF, sf_half);
       float l_tile = 0.0f;
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
@@ -417,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
               TMEM_ST8(t_oc, oc);
             }
           }
-          *reinterpret_cast<uint4*>(sP + tile_code_offset(row, kBlocksPerThread * h + b)) = w;
+          sts128(b == 0 ? aP0 : aP1, w);
           if (!kPnq) l_tile = fmaf(sx, sigma[b], l_tile);   // Eq. 12
         }
         if (kResc) {
@@ -442,11 +437,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     // ---- epilogue: O = O~ / l (line 18) ----
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
     float l = l_run;
-    if (!kPnq && kSplit == 2) {                    // add the partner's half of the row sum
-      float* mslot = sMax + ((T & 1) * 2 + t) * 256;
-      mslot[h * 128 + row] = l_run;
+    if (!kPnq) {                                   // add the partner's half of the row sum
+      const uint32_t par = (uint32_t)(T & 1) * 2048u;
+      sts32f(aMaxOwn + par, l_run);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-      l = l_run + mslot[(h ^ 1) * 128 + row];
+      l = l_run + lds32f(aMaxPartner + par);
     }
     if (ok) {
       tc_fence_after();
