@@ -28,62 +28,46 @@ __device__ __forceinline__ uint32_t quantize_bf16x8(const uint4& v, float inv) {
                      bf16lo(v.z) * inv, bf16hi(v.z) * inv, bf16lo(v.w) * inv, bf16hi(v.w) * inv);
 }
 
-// Fixed Hadamard rotation of one 128-element row held by 16 consecutive lanes, 8 elements per lane
-// (element index = 8 * (lane % 16) + i): y = x H_128 / sqrt(128) (paper Algorithm 2, lines 1-2).
-// Fast Walsh-Hadamard butterfly in fp32, strides 1, 2, 4 inside the thread and 8, 16, 32, 64 across
-// lanes, every stage (a, b) -> (a + b, a - b) with a the lower index, then one multiply by
-// fl32(1/sqrt(128)).  The stage order and the fp32 arithmetic are part of the definition, because
-// the result feeds a rounding decision; __fadd_rn / __fsub_rn keep the compiler from contracting.
-__device__ __forceinline__ void hadamard128_rows(float (&f)[8], int lane) {
-#pragma unroll
-  for (int s = 1; s < 8; s <<= 1) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if ((i & s) == 0) {
-        const float a = f[i], b = f[i + s];
-        f[i] = __fadd_rn(a, b);
-        f[i + s] = __fsub_rn(a, b);
-      }
-    }
-  }
-#pragma unroll
-  for (int m = 1; m < 16; m <<= 1) {
-    const bool upper = (lane & m) != 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float other = __shfl_xor_sync(0xFFFFFFFFu, f[i], m);
-      f[i] = upper ? __fsub_rn(other, f[i]) : __fadd_rn(f[i], other);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) f[i] = __fmul_rn(f[i], 0.08838834764831845f);
+// Packed fp32x2 arithmetic (two IEEE round-to-nearest fp32 operations per instruction; each half gives
+// exactly the result of the scalar instruction).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
 }
 
 // One 16-byte chunk (8 bf16) -> packed codes and the block's shared exponent; the four lanes of a
-// 32-element block combine their maxima with two shuffles.  With kRotate the 16 lanes of a row
-// first apply the Hadamard rotation and the block maximum is taken on the fp32 results.
-template <bool kRotate>
-__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, int lane, uint32_t rule, int* e_out) {
-  if (kRotate) {
-    float f[8] = {bf16lo(v.x), bf16hi(v.x), bf16lo(v.y), bf16hi(v.y), bf16lo(v.z), bf16hi(v.z), bf16lo(v.w), bf16hi(v.w)};
-    hadamard128_rows(f, lane);
-    uint32_t m = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) m = max(m, __float_as_uint(f[i]) & 0x7FFFFFFFu);
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-    const int e = shared_exponent_rule(m, rule);
-    const float inv = pow2_neg(e);
-    *e_out = e;
-    return pack_e2m1x8(f[0] * inv, f[1] * inv, f[2] * inv, f[3] * inv, f[4] * inv, f[5] * inv, f[6] * inv, f[7] * inv);
-  } else {
-    uint32_t m = absmax_bf16x8(v);
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-    const int e = shared_exponent_rule(m << 16, rule);
-    *e_out = e;
-    return quantize_bf16x8(v, pow2_neg(e));
-  }
+// 32-element block combine their maxima with two shuffles.
+__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, uint32_t rule, int* e_out) {
+  uint32_t m = absmax_bf16x8(v);
+  m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+  m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+  const int e = shared_exponent_rule(m << 16, rule);
+  *e_out = e;
+  return quantize_bf16x8(v, pow2_neg(e));
 }
 
 constexpr int kQThreads = 256;
@@ -94,7 +78,6 @@ constexpr int kQThreads = 256;
 // consecutive chunks (32 KiB) and issues all of its loads before it quantizes anything.
 constexpr int kQChunksPerThread = 8;
 
-template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t n_chunks, uint32_t rule) {
@@ -110,7 +93,7 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
   for (int u = 0; u < kQChunksPerThread; ++u) {
     const int64_t i = base + u * kQThreads;
     int e;
-    const uint32_t packed = quantize_chunk<kRotate>(v[u], lane, rule, &e);
+    const uint32_t packed = quantize_chunk(v[u], rule, &e);
     // four consecutive blocks (16 lanes) -> one 32-bit scale word
     const uint32_t eb = (uint32_t)(e + 127);
     const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
@@ -136,7 +119,6 @@ quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes
 // tile: 32 KiB in, 8.5 KiB out.  A thread issues its eight 16-byte loads up front (the whole
 // tile is in flight at once), then quantizes them; a warp covers two full rows per step, so the
 // four lanes of a block and the sixteen lanes of a row are always in the same warp.
-template <bool kRotate>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
                            uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
@@ -158,7 +140,7 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
     const int chunk = k * kQThreads + tid;
     const int r = chunk >> 4, c = (chunk >> 2) & 3;
     int e;
-    const uint32_t packed = quantize_chunk<kRotate>(v[k], lane, rule, &e);
+    const uint32_t packed = quantize_chunk(v[k], rule, &e);
     const uint32_t eb = (uint32_t)(e + 127);
     const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
     const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
@@ -166,6 +148,117 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
     ctile[tile_code_offset(r, c) / 4 + (chunk & 3)] = packed;
     if ((lane & 15) == 0)
       *reinterpret_cast<uint32_t*>(stile + tile_scale_offset(r, 0)) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Axis 1 with the Hadamard rotation (cols == 128), both layouts.  A CTA takes 128 consecutive rows;
+// FOUR lanes share a row and each holds 32 of its elements: lane q (0..3) loads the 16-byte chunks
+// q, q + 4, q + 8, q + 12, so element index = 32 u + 8 q + i with u = 0..3 the chunk number within the
+// lane and i = 0..7.  The butterfly stages of strides 1, 2, 4 (bits of i) and 32, 64 (bits of u) stay
+// inside the thread; only strides 8 and 16 (bits of q) cross lanes -- two shuffle stages per row
+// instead of the four that an 8-elements-per-lane split needs.  Stage order (ascending strides) and
+// the fp32 arithmetic (every stage (a, b) -> (a + b, a - b) with a the lower index, then one multiply by
+// fl32(1/sqrt(128))) are part of the definition, because the result feeds a rounding decision.  The MX block
+// u is the chunk u of the four lanes: its maximum takes two more shuffles, its codes are one word per
+// lane, its scale byte is written (with the row's other three) by lane 0.
+template <bool kTileLayout>
+__global__ void __launch_bounds__(kQThreads)
+quantize_axis1_rot_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
+                          uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
+  const int tid = threadIdx.x;
+  const int q = tid & 3, rr = tid >> 2;              // lane within the row's quad; row within a 64-row pass
+  // tile layout: grid = (row tiles, batch), `rows` per batch entry; canonical: grid = row groups, `rows` in total
+  const int64_t row0 = (int64_t)blockIdx.x * kTile;
+  const uint4* src = in + ((kTileLayout ? (int64_t)blockIdx.y * rows : 0) + row0) * 16;     // 16 chunks per row
+  const int rows_here = (int)min((int64_t)kTile, rows - row0);
+  uint4 v[2][4];
+#pragma unroll
+  for (int k = 0; k < 2; ++k)
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = k * 64 + rr;
+      v[k][u] = r < rows_here ? __ldg(src + r * 16 + 4 * u + q) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  const int64_t tile = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+  const uint64_t sgn1 = (q & 1) ? pack2(-1.0f, -1.0f) : pack2(1.0f, 1.0f);
+  const uint64_t sgn2 = (q & 2) ? pack2(-1.0f, -1.0f) : pack2(1.0f, 1.0f);
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int r = k * 64 + rr;
+    // the 32 values as 16 packed pairs: pair j = elements (2j, 2j + 1) of the thread
+    uint64_t pr[16];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint4& w = v[k][u];
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        // stride 1 on the way in: (a, b) -> (a + b, a - b)
+        const float a = bf16lo(ww[j]), b = bf16hi(ww[j]);
+        pr[4 * u + j] = pack2(__fadd_rn(a, b), __fsub_rn(a, b));
+      }
+    }
+    // strides 2, 4 (pair strides 1, 2): inside each chunk, two elements per instruction
+#pragma unroll
+    for (int st = 1; st < 4; st <<= 1)
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if ((j & st) == 0) {
+          const uint64_t a = pr[j], b = pr[j + st];
+          pr[j] = add2(a, b);
+          pr[j + st] = sub2(a, b);
+        }
+    // strides 8, 16: across the quad.  The lower lane gets a + b = own * 1 + other, the upper one
+    // a - b = own * (-1) + other (the product is exact, so the fma rounds like the add / subtract).
+#pragma unroll
+    for (int j = 0; j < 16; ++j) pr[j] = fma2(pr[j], sgn1, __shfl_xor_sync(0xFFFFFFFFu, pr[j], 1));
+#pragma unroll
+    for (int j = 0; j < 16; ++j) pr[j] = fma2(pr[j], sgn2, __shfl_xor_sync(0xFFFFFFFFu, pr[j], 2));
+    // strides 32, 64 (pair strides 4, 8): across the thread's chunks
+#pragma unroll
+    for (int st = 4; st < 16; st <<= 1)
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if ((j & st) == 0) {
+          const uint64_t a = pr[j], b = pr[j + st];
+          pr[j] = add2(a, b);
+          pr[j + st] = sub2(a, b);
+        }
+    uint32_t word[4], sf = 0;
+    const uint64_t norm2 = pack2(0.08838834764831845f, 0.08838834764831845f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float mf = 0.0f;                               // max |.| as a float: the operand modifiers make |x| free
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        pr[4 * u + j] = mul2(pr[4 * u + j], norm2);
+        float lo, hi;
+        unpack2(pr[4 * u + j], lo, hi);
+        mf = fmaxf(fmaxf(mf, fabsf(lo)), fabsf(hi));
+      }
+      mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 1));
+      mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 2));
+      const int e = shared_exponent_rule(__float_as_uint(mf), rule);
+      const float inv = pow2_neg(e);
+      const uint64_t inv2 = pack2(inv, inv);
+      float x[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) unpack2(mul2(pr[4 * u + j], inv2), x[2 * j], x[2 * j + 1]);
+      word[u] = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+      sf |= (uint32_t)(e + 127) << (8 * u);
+    }
+    if (kTileLayout) {
+      uint32_t* ctile = reinterpret_cast<uint32_t*>(codes + tile * kTileCodeBytes);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) ctile[tile_code_offset(r, u) / 4 + q] = word[u];
+      if (q == 0) *reinterpret_cast<uint32_t*>(scales + tile * kTileScaleBytes + tile_scale_offset(r, 0)) = sf;
+    } else if (r < rows_here) {
+      uint32_t* crow = reinterpret_cast<uint32_t*>(codes) + (row0 + r) * 16;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) crow[4 * u + q] = word[u];
+      if (q == 0) *reinterpret_cast<uint32_t*>(scales + (row0 + r) * 4) = sf;
+    }
   }
 }
 
@@ -289,17 +382,19 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
       if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
       if (rotate)
-        quantize_axis1_tile_kernel<true><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
-                                                                         (uint8_t*)scales, rows, rule);
+        quantize_axis1_rot_kernel<true><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
+                                                                        (uint8_t*)scales, rows, rule);
       else
-        quantize_axis1_tile_kernel<false><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
+        quantize_axis1_tile_kernel<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
                                                                           (uint8_t*)scales, rows, rule);
     } else {
-      if (rotate)
-        quantize_axis1_kernel<true><<<(unsigned)blocks, kQThreads, 0, stream>>>(
-            (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
-      else
-        quantize_axis1_kernel<false><<<(unsigned)blocks, kQThreads, 0, stream>>>(
+      if (rotate) {                                  // cols == 128 here: batch * rows rows of 16 chunks
+        const int64_t groups = (batch * rows + kTile - 1) / kTile;
+        if (groups > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
+        quantize_axis1_rot_kernel<false><<<(unsigned)groups, kQThreads, 0, stream>>>(
+            (const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, batch * rows, rule);
+      } else
+        quantize_axis1_kernel<<<(unsigned)blocks, kQThreads, 0, stream>>>(
             (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
     }
   } else {
