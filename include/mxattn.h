@@ -147,6 +147,26 @@ int mxattn_forward_prequantized(const void* q_codes, const void* q_scales,
                                 int B, int H, int64_t Nq, int64_t Nkv, int d,
                                 float softmax_scale, unsigned flags, void* status, void* stream);
 
+/* Debugging aid for small problems: mxattn_forward_ws that also writes out what the softmax loop
+ * produced, so that Algorithm 2 lines 10-14 can be checked tile by tile (the quantized probabilities
+ * P-hat code for code, the running maxima and the final row sums) instead of only through O.
+ * flags must contain MXATTN_FLAG_OUT_FP32.  `dump` is caller-owned device memory of at least
+ * mxattn_forward_debug_dump_bytes() bytes (MXATTN_EWORKSPACE if smaller, MXATTN_EUNSUPPORTED above
+ * 1 GiB), 16-byte aligned, laid out as
+ *   [B*H][query tiles][KV tiles] records of 9216 bytes:
+ *        8192 bytes  P-hat codes of the 128 x 128 tile, MXATTN_LAYOUT_TILE image (rows = queries,
+ *                    blocks of 32 along the keys)
+ *         512 bytes  its E8M0 scales, MXATTN_LAYOUT_TILE scale atom
+ *         512 bytes  128 fp32: the running maximum m after this KV tile, per query row of the tile
+ *   then [B*H][query tiles][128] fp32: the final row sum l (Algorithm 2 line 14) per query row.
+ * Rows beyond Nq and columns beyond Nkv hold the values of the zero padding (code 0). */
+size_t mxattn_forward_debug_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);
+int mxattn_forward_debug_dump(const void* q, const void* k, const void* v, void* o,
+                              int B, int H, int64_t Nq, int64_t Nkv, int d,
+                              float softmax_scale, unsigned flags,
+                              void* workspace, size_t workspace_bytes,
+                              void* dump, size_t dump_bytes, void* stream);
+
 /* bf16 variant of the same fused kernel, with no quantization anywhere: the FlashAttention-2
  * recurrence the paper starts from (Section 2, Eq. 2-3) with bf16 operands on the tensor cores, the
  * exponentials rounded to bf16 for the second GEMM and the row sum taken from the fp32 exponentials.

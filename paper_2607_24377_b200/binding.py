@@ -49,6 +49,9 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
         L.mxattn_forward_static.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
         L.mxattn_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
+        L.mxattn_forward_debug_dump_bytes.argtypes = [ci, ci, i64, i64, ci]
+        L.mxattn_forward_debug_dump_bytes.restype = sz
+        L.mxattn_forward_debug_dump.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp, sz, vp]
         L.mxattn_forward_bf16_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_bf16_workspace_bytes.restype = sz
         L.mxattn_forward_bf16.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
@@ -128,6 +131,17 @@ def forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):
                                    flags, _ptr(workspace),
                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
                                    _stream()), "mxattn_forward_ws")
+
+
+def forward_debug_dump_bytes(B, H, Nq, Nkv, d) -> int:
+    return int(lib().mxattn_forward_debug_dump_bytes(B, H, Nq, Nkv, d))
+
+
+def forward_debug_dump(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, dump):
+    _check(lib().mxattn_forward_debug_dump(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d, softmax_scale, flags,
+                                           _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                           _ptr(dump), 0 if dump is None else dump.numel() * dump.element_size(), _stream()),
+           "mxattn_forward_debug_dump")
 
 
 def forward_bf16_workspace_bytes(B, H, Nq, Nkv, d) -> int:

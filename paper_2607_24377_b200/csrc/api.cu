@@ -37,7 +37,7 @@ static bool carve(int B, int H, int64_t Nq, int64_t Nkv, int d, WorkspaceLayout*
 
 static int forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq,
                       int64_t Nkv, int d, float softmax_scale, unsigned flags, void* workspace,
-                      size_t workspace_bytes, cudaStream_t stream) {
+                      size_t workspace_bytes, cudaStream_t stream, void* dump = nullptr) {
   if (!q || !k || !v || !o) return MXATTN_EINVAL;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
   if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32 | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
@@ -62,7 +62,7 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
   // lines 6-19
   return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
                         ws + w.v_scales, o, B, H, Nq, Nkv, softmax_scale, flags,
-                        reinterpret_cast<int*>(ws + w.status), stream);
+                        reinterpret_cast<int*>(ws + w.status), stream, dump);
 }
 
 }  // namespace mxattn
@@ -93,6 +93,27 @@ extern "C" int mxattn_forward_ws(const void* q, const void* k, const void* v, vo
                                  void* workspace, size_t workspace_bytes, void* stream) {
   return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, workspace_bytes,
                     (cudaStream_t)stream);
+}
+
+extern "C" size_t mxattn_forward_debug_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || d != kHeadDim) return 0;
+  return forward_dump_bytes(B, H, Nq, Nkv);
+}
+
+extern "C" int mxattn_forward_debug_dump(const void* q, const void* k, const void* v, void* o, int B, int H,
+                                         int64_t Nq, int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                                         void* workspace, size_t workspace_bytes, void* dump,
+                                         size_t dump_bytes, void* stream) {
+  if (!dump) return MXATTN_EINVAL;
+  if (!(flags & MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  const size_t need = forward_dump_bytes(B, H, Nq, Nkv);
+  if (need > ((size_t)1 << 30)) return MXATTN_EUNSUPPORTED;      // a debugging aid for small problems
+  if (dump_bytes < need) return MXATTN_EWORKSPACE;
+  if (!aligned16(dump)) return MXATTN_EALIGN;
+  return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, workspace_bytes,
+                    (cudaStream_t)stream, dump);
 }
 
 extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_scales, const void* k_codes,

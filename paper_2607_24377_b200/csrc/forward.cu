@@ -55,6 +55,7 @@ constexpr int kThreads = 32 * (kSoftmaxWarps + 2);   // softmax warps + producer
 constexpr int kStages = 4;
 constexpr int kNV = 144;                         // GEMM 2 N: 128 channels + 16 rows of ones
 constexpr int kVStageBytes = kNV * 64;           // 9216
+constexpr int kDumpTileBytes = kTileCodeBytes + kTileScaleBytes + kTile * 4;   // debug dump: codes, scale atom, m per row
 
 // shared memory map (byte offsets from a 1024-aligned base)
 constexpr int kOffQ = 0;                                   // 2 x 8192
@@ -100,13 +101,15 @@ struct Params {
   const uint8_t* v_codes; const uint8_t* v_scales;
   void* out;
   int* status;
+  uint8_t* dump;        // per-tile P-hat images, scales, running maxima and final row sums (debug entry point only)
   int64_t Nq, Nkv;
   int q_tiles, kv_tiles, q_pairs;
   float scale_log2e;    // softmax_scale * log2(e)
+  float softmax_scale;
 };
 
 // ---------------------------------------------------------------------------------------------
-template <bool kUos, bool kPnq, bool kOutF32>
+template <bool kUos, bool kPnq, bool kOutF32, bool kDump>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -385,6 +388,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       }
       // the scale bytes go out before the exponentials, so only the code stores precede the proxy fence
       sts16(aSF, sf_half);
+      uint8_t* dump_tile = nullptr;
+      if (kDump && 2 * pair + t < p.q_tiles) {       // image of this (query tile, KV tile): codes, scale atom, m
+        dump_tile = p.dump + ((((int64_t)bh * p.q_tiles + 2 * pair + t) * T) + j) * kDumpTileBytes;
+        *reinterpret_cast<uint16_t*>(dump_tile + kTileCodeBytes + tile_scale_offset(row, 2 * h)) = (uint16_t)sf_half;
+        if (h == 0) reinterpret_cast<float*>(dump_tile + kTileCodeBytes + kTileScaleBytes)[row] = m_new * p.softmax_scale;   // the kernel keeps m in unscaled score units
+      }
       float l_tile = 0.0f;
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
@@ -413,6 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
             }
           }
           sts128(b == 0 ? aP0 : aP1, w);
+          if (kDump && dump_tile) *reinterpret_cast<uint4*>(dump_tile + tile_code_offset(row, kBlocksPerThread * h + b)) = w;
           if (!kPnq) l_tile = fmaf(sx, sigma[b], l_tile);   // Eq. 12
         }
         if (kResc) {
@@ -454,6 +464,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         l = __uint_as_float(lr);
       }
       const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
+      if (kDump && h == 0 && qtile < p.q_tiles)
+        reinterpret_cast<float*>(p.dump + (int64_t)gridDim.x / p.q_pairs * p.q_tiles * T * kDumpTileBytes)
+            [((int64_t)bh * p.q_tiles + qtile) * kTile + row] = l;
       const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + kCols * h;
 #pragma unroll 1
       for (int c0 = 0; c0 < kCols; c0 += 32) {
@@ -516,28 +529,40 @@ int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
 }
 
+size_t forward_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv) {
+  const int64_t qt = (Nq + kTile - 1) / kTile, kt = (Nkv + kTile - 1) / kTile;
+  return (size_t)((int64_t)B * H * qt * kt * fwd::kDumpTileBytes + (int64_t)B * H * qt * kTile * 4);
+}
+
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes, const void* k_scales,
                    const void* v_codes, const void* v_scales, void* o, int B, int H, int64_t Nq, int64_t Nkv,
-                   float softmax_scale, unsigned flags, int* status, cudaStream_t stream) {
+                   float softmax_scale, unsigned flags, int* status, cudaStream_t stream, void* dump) {
   using namespace fwd;
   Params p;
   p.q_codes = (const uint8_t*)q_codes; p.q_scales = (const uint8_t*)q_scales;
   p.k_codes = (const uint8_t*)k_codes; p.k_scales = (const uint8_t*)k_scales;
   p.v_codes = (const uint8_t*)v_codes; p.v_scales = (const uint8_t*)v_scales;
-  p.out = o; p.status = status; p.Nq = Nq; p.Nkv = Nkv;
+  p.out = o; p.status = status; p.dump = (uint8_t*)dump; p.Nq = Nq; p.Nkv = Nkv;
   const int64_t qt = (Nq + kTile - 1) / kTile, kt = (Nkv + kTile - 1) / kTile;
   const int64_t pairs = (qt + 1) / 2;
   const int64_t grid = (int64_t)B * H * pairs;
   if (qt > 0x3FFFFFFF || kt > 0x3FFFFFFF || grid > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
   p.q_tiles = (int)qt; p.kv_tiles = (int)kt; p.q_pairs = (int)pairs;
   p.scale_log2e = softmax_scale * 1.4426950408889634f;
+  p.softmax_scale = softmax_scale;
 
   const bool uos = flags & MXATTN_FLAG_UOS, pnq = flags & MXATTN_FLAG_PNQ, f32 = flags & MXATTN_FLAG_OUT_FP32;
   void (*kern)(const Params) = nullptr;
-#define PICK(U, P, F) if (uos == U && pnq == P && f32 == F) kern = attention_kernel<U, P, F>;
+#define PICK(U, P, F) if (uos == U && pnq == P && f32 == F) kern = attention_kernel<U, P, F, false>;
   PICK(false, false, false) PICK(false, false, true) PICK(false, true, false) PICK(false, true, true)
   PICK(true, false, false) PICK(true, false, true) PICK(true, true, false) PICK(true, true, true)
 #undef PICK
+  if (dump) {                                     // debug entry point: fp32 output only
+    if (!f32) return MXATTN_EINVAL;
+#define PICKD(U, P) if (uos == U && pnq == P) kern = attention_kernel<U, P, true, true>;
+    PICKD(false, false) PICKD(false, true) PICKD(true, false) PICKD(true, true)
+#undef PICKD
+  }
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return MXATTN_ECUDA;
   kern<<<(unsigned)grid, kThreads, kSmemBytes, stream>>>(p);

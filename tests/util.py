@@ -51,3 +51,23 @@ def canonical_to_tile_axis0(codes: np.ndarray, scales: np.ndarray):
                 tc[t, off + b] = codes[n, t * 64 + c * 16 + b]
             ts[t, tile_scale_offset(n, c)] = scales[n, t * 4 + c]
     return tc, ts
+
+
+E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def decode_tile_axis1(tile_codes: np.ndarray, tile_scales: np.ndarray) -> np.ndarray:
+    """One 8192-byte tile image + its 512-byte scale atom -> the [128, 128] float64 values it encodes
+    (rows x 128 elements, blocks of 32 along the row).  Pure byte shuffling plus the E2M1 / E8M0 tables."""
+    r = np.arange(128)
+    out = np.zeros((128, 128))
+    for c in range(4):
+        off = tile_code_offset(r, c)
+        byts = np.stack([tile_codes[off + b] for b in range(16)], axis=1)        # [128, 16]
+        nib = np.empty((128, 32), np.uint8)
+        nib[:, 0::2] = byts & 15
+        nib[:, 1::2] = byts >> 4
+        val = E2M1_VALUES[nib & 7] * np.where(nib & 8, -1.0, 1.0)
+        e = tile_scales[tile_scale_offset(r, c)].astype(np.int32) - 127
+        out[:, 32 * c:32 * c + 32] = np.ldexp(val, e[:, None])
+    return out
