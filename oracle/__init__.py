@@ -12,6 +12,8 @@ Modules
 ``attention``  tiled online-softmax forward with direct or pre-normalization placement of the
                P-tilde quantizer (Section 2 recurrence, Eq. 12, Eq. 22, Algorithm 2), and the
                float64 dense softmax attention.
+``rowsum``     the row-sum diagnostic of Section 5.3: quantize materialized probabilities, split the row-sum
+               error into zeroing / saturation / downward / upward rounding, and the row entropy.
 ``uos_theory`` the quantization-error objective E, D, Delta, J of Section 4.1 / Appendices B-C,
                evaluated numerically; used to pin the 7.25 boundary independently of the quantizer.
 
