@@ -7,6 +7,8 @@
   OCP direct, UOS direct, UOS+PNQ, UOS+PNQ+Hadamard}: kernel-only ms / TFLOP/s, whole-step ms, and the
   relative L2 error against float64 dense attention on sampled rows (CPU oracle);
 * outlier config (H=24, N=8192): the same quality comparison;
+* row-sum diagnostic (Section 5.3): mean row sum of the quantized materialized probabilities and its split
+  by quantization outcome, OCP / UOS / UOS+Hadamard, on three synthetic recipes at N=4096;
 * quantize: 2^20 .. 2^29 bf16 elements, axis 1 and axis 0, OCP and UOS: GB/s and fraction of the
   measured HBM copy rate.
 
@@ -85,6 +87,26 @@ def main():
         torch.cuda.empty_cache()
     doc["outlier_config"] = attention_report(si.CONFIGS["outlier"], heads_for_quality=(0, 7, 15, 23), rows_per_head=16)
     torch.cuda.empty_cache()
+
+    # row-sum diagnostic of Section 5.3 on synthetic rows (means over all rows of the config)
+    doc["rowsum_diagnostic"] = []
+    for name, cfg in (("iid N=4096", si.custom_config("iid4096", 1, 8, 4096, 4096, 11)),
+                      ("wan recipe N=4096", si.custom_config("wan4096", 1, 8, 4096, 4096, 12, "wan")),
+                      ("outlier recipe N=4096", si.CONFIGS["sweep4096"])):
+        q, k, _ = si.make_all(cfg)
+        dq, dk = dev(q), dev(k)
+        out6 = torch.empty((cfg.B, cfg.H, cfg.Nq, 6), dtype=torch.float32, device="cuda")
+        ws = torch.empty(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), dtype=torch.uint8, device="cuda")
+        for label, fl in (("ocp", 0), ("uos", mx.FLAG_UOS), ("uos_hadamard", mx.FLAG_UOS | mx.FLAG_HADAMARD)):
+            ms = timed(lambda: mx.rowsum_diagnostic(dq, dk, out6, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, fl, ws))
+            assert mx.device_status(ws) == 0
+            o = out6.double().cpu().numpy().reshape(-1, 6)
+            doc["rowsum_diagnostic"].append({
+                "data": name, "rule": label, "ms": ms, "mean_row_sum": float(o[:, 0].mean()),
+                "zeroing": float(o[:, 1].mean()), "saturation": float(o[:, 2].mean()), "downward": float(o[:, 3].mean()),
+                "upward": float(o[:, 4].mean()), "mean_entropy": float(o[:, 5].mean()),
+                "frac_rows_under_normalized": float((o[:, 0] < 1.0).mean())})
+        torch.cuda.empty_cache()
 
     exps = (20, 24) if args.quick else range(20, 30)
     for e in exps:

@@ -167,6 +167,25 @@ int mxattn_forward_debug_dump(const void* q, const void* k, const void* v, void*
                               void* workspace, size_t workspace_bytes,
                               void* dump, size_t dump_bytes, void* stream);
 
+/* Row-sum diagnostic of MXFP4 probability quantization (paper Section 5.3, figure "Row-sum
+ * diagnostics", panels A, B, D).  Per query row: P = softmax(Q-hat K-hat^T * softmax_scale) as if
+ * materialized (Q, K quantized as in mxattn_forward, same rule), rounded to fp32 and quantized in
+ * 32-blocks along the keys; out receives six fp32 per row:
+ *   [0] the row sum of the quantized probabilities (1 would be exact normalization),
+ *   [1] the part of (row sum - 1) due to non-zero probabilities that quantize to zero,
+ *   [2] ... due to saturation (scaled value above the largest E2M1 value 6),
+ *   [3] ... due to downward rounding of the remaining elements,  [4] ... due to upward rounding,
+ *   [5] the row's entropy -sum p ln p.
+ * q: [B,H,Nq,d], k: [B,H,Nkv,d] bf16 device pointers; out: [B,H,Nq,6] fp32 device pointer; d = 128.
+ * flags: MXATTN_FLAG_UOS (rule for Q, K and P; otherwise the OCP rule), MXATTN_FLAG_HADAMARD.
+ * workspace: at least mxattn_forward_workspace_bytes(B,H,Nq,Nkv,d) bytes (holds Q-hat, K-hat and the
+ * status word read by mxattn_device_status).  The scores are computed twice by the FP4 tensor-core
+ * GEMM of the attention kernel; nothing of size Nq x Nkv is stored.  Same error codes as mxattn_forward_ws. */
+int mxattn_rowsum_diagnostic(const void* q, const void* k, void* out,
+                             int B, int H, int64_t Nq, int64_t Nkv, int d,
+                             float softmax_scale, unsigned flags,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
 /* bf16 variant of the same fused kernel, with no quantization anywhere: the FlashAttention-2
  * recurrence the paper starts from (Section 2, Eq. 2-3) with bf16 operands on the tensor cores, the
  * exponentials rounded to bf16 for the second GEMM and the row sum taken from the fp32 exponentials.

@@ -49,6 +49,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
         L.mxattn_forward_static.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp]
         L.mxattn_forward_ws.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
+        L.mxattn_rowsum_diagnostic.argtypes = [vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
         L.mxattn_forward_debug_dump_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_debug_dump_bytes.restype = sz
         L.mxattn_forward_debug_dump.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp, sz, vp]
@@ -131,6 +132,12 @@ def forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):
                                    flags, _ptr(workspace),
                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
                                    _stream()), "mxattn_forward_ws")
+
+
+def rowsum_diagnostic(q, k, out, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):
+    _check(lib().mxattn_rowsum_diagnostic(_ptr(q), _ptr(k), _ptr(out), B, H, Nq, Nkv, d, softmax_scale, flags,
+                                          _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                          _stream()), "mxattn_rowsum_diagnostic")
 
 
 def forward_debug_dump_bytes(B, H, Nq, Nkv, d) -> int:

@@ -95,6 +95,34 @@ extern "C" int mxattn_forward_ws(const void* q, const void* k, const void* v, vo
                     (cudaStream_t)stream);
 }
 
+extern "C" int mxattn_rowsum_diagnostic(const void* q, const void* k, void* out, int B, int H, int64_t Nq,
+                                        int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                                        void* workspace, size_t workspace_bytes, void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!q || !k || !out) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(out)) return MXATTN_EALIGN;
+  WorkspaceLayout w;
+  if (!carve(B, H, Nq, Nkv, d, &w)) return MXATTN_EUNSUPPORTED;
+  if (!workspace || workspace_bytes < w.total) return MXATTN_EWORKSPACE;
+  if (!aligned16(workspace)) return MXATTN_EALIGN;
+  g_launches = 0;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const int mode = (flags & MXATTN_FLAG_UOS) ? MXATTN_MODE_UOS : MXATTN_MODE_OCP;
+  const int qk_mode = mode | ((flags & MXATTN_FLAG_HADAMARD) ? MXATTN_MODE_HADAMARD : 0);
+  const int64_t bh = (int64_t)B * H;
+  if (cudaMemsetAsync(ws + w.status, 0, 16, stream) != cudaSuccess) return MXATTN_ECUDA;
+  int rc;
+  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  return launch_rowsum_diag(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, out, B, H, Nq, Nkv,
+                            softmax_scale, (flags & MXATTN_FLAG_UOS) ? kRuleUos : kRuleOcp,
+                            reinterpret_cast<int*>(ws + w.status), stream);
+}
+
 extern "C" size_t mxattn_forward_debug_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d) {
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || d != kHeadDim) return 0;
   return forward_dump_bytes(B, H, Nq, Nkv);

@@ -81,20 +81,6 @@ enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages, BAR_VFULL
 constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK = 424,
                    kColSFV = 432, kColSFP = 448;
 
-// ---------------------------------------------------------------------------------------------
-// instruction descriptor of kind::mxf4.block_scale: A, B = E2M1 (K-major), scales UE8M0, M = 128
-__device__ __forceinline__ constexpr uint32_t make_idesc(int n, int ks) {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
-         ((uint32_t)(ks * 2) << 29) | ((uint32_t)(ks * 2) << 4);
-}
-
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb) : "memory");
-}
-
 struct Params {
   const uint8_t* q_codes; const uint8_t* q_scales;
   const uint8_t* k_codes; const uint8_t* k_scales;
