@@ -162,7 +162,9 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
 // fl32(1/sqrt(128))) are part of the definition, because the result feeds a rounding decision.  The MX block
 // u is the chunk u of the four lanes: its maximum takes two more shuffles, its codes are one word per
 // lane, its scale byte is written (with the row's other three) by lane 0.
-template <bool kTileLayout>
+// kRuleKind: 0 = OCP floor rule, 1 = UOS (boundary 7.25, the mantissa compare of shared_exponent), 2 = the
+// boundary passed in `rule` (this kernel is bound by instruction issue, so the common rules are compiled in).
+template <bool kTileLayout, int kRuleKind>
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_rot_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
                           uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
@@ -239,7 +241,8 @@ quantize_axis1_rot_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ co
       }
       mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 1));
       mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 2));
-      const int e = shared_exponent_rule(__float_as_uint(mf), rule);
+      const int e = kRuleKind == 2 ? shared_exponent_ceil(__float_as_uint(mf), rule)
+                                   : shared_exponent(__float_as_uint(mf), kRuleKind == 1);
       const float inv = pow2_neg(e);
       const uint64_t inv2 = pack2(inv, inv);
       float x[8];
@@ -381,18 +384,21 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
     if (tile) {
       if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
-      if (rotate)
-        quantize_axis1_rot_kernel<true><<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
-                                                                        (uint8_t*)scales, rows, rule);
-      else
+      if (rotate) {
+        auto kern = rule == kRuleOcp ? quantize_axis1_rot_kernel<true, 0>
+                  : rule == kRuleUos ? quantize_axis1_rot_kernel<true, 1> : quantize_axis1_rot_kernel<true, 2>;
+        kern<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, rows, rule);
+      } else
         quantize_axis1_tile_kernel<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
                                                                           (uint8_t*)scales, rows, rule);
     } else {
       if (rotate) {                                  // cols == 128 here: batch * rows rows of 16 chunks
         const int64_t groups = (batch * rows + kTile - 1) / kTile;
         if (groups > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
-        quantize_axis1_rot_kernel<false><<<(unsigned)groups, kQThreads, 0, stream>>>(
-            (const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, batch * rows, rule);
+        auto kern = rule == kRuleOcp ? quantize_axis1_rot_kernel<false, 0>
+                  : rule == kRuleUos ? quantize_axis1_rot_kernel<false, 1> : quantize_axis1_rot_kernel<false, 2>;
+        kern<<<(unsigned)groups, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales,
+                                                         batch * rows, rule);
       } else
         quantize_axis1_kernel<<<(unsigned)blocks, kQThreads, 0, stream>>>(
             (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
