@@ -122,7 +122,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     mbar_init(bar(BAR_SFREE), 4 * kSplit);                  // one arrival per softmax warp of the draining group
     mbar_init(bar(BAR_PFULL + 0), 4 * kSplit); mbar_init(bar(BAR_PFULL + 1), 4 * kSplit);   // one arrival per softmax warp
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
-    *abort_flag = 0;
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // constant rows of ones appended to every V stage (E2M1 code 2 = 1.0) and their scale atom (2^0)
@@ -290,10 +291,16 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     const uint32_t aMaxOwn = sbase + kOffMax + (t * 256 + h * 128 + row) * 4;
     const uint32_t aMaxPartner = sbase + kOffMax + (t * 256 + (h ^ 1) * 128 + row) * 4;
     const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
+    // The two warps of a pair meet at an (unbounded) named barrier in every tile, so they must take the same
+    // decision at every bounded wait before it.  Both always wait on the same mbarrier; they therefore give up
+    // only on their own cycle limit, never because another role of the CTA raised the abort flag (a warp that
+    // saw the flag could leave while its partner, a moment later, finds the barrier complete and goes on to
+    // the pair barrier alone).  Their waits watch a flag that nothing sets, and raise the CTA's flag on expiry.
+    volatile int* const own_limit_only = abort_flag + 1;
     bool ok = true;
 
     for (int j = 0; j < T; ++j) {
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[kCols];
@@ -339,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       m_run = m_new;
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), abort_flag, p.status, 32));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
         if (!ok) break;
       }
       tc_fence_after();
@@ -431,7 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     }
 
     // ---- epilogue: O = O~ / l (line 18) ----
-    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     float l = l_run;
     if (!kPnq) {                                   // add the partner's half of the row sum
       const uint32_t par = (uint32_t)(T & 1) * 2048u;

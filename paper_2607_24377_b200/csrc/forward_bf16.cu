@@ -132,7 +132,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
     mbar_init(bar(BAR_SFREE), 8);
     mbar_init(bar(BAR_PFULL + 0), 8); mbar_init(bar(BAR_PFULL + 1), 8);
     mbar_init(bar(BAR_ODONE + 0), 1); mbar_init(bar(BAR_ODONE + 1), 1);
-    *abort_flag = 0;
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == kSoftmaxWarps + 1) {
@@ -267,10 +268,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
     uint8_t* sP = smem + kOffP + t * kTileBytes + h * kHalfBytes;       // this thread's keys are one K half of P
     float* sMax = reinterpret_cast<float*>(smem + kOffMax) + t * 256;
     const int pair_bar = 1 + (warp & 3) + 4 * t;
+    // the two warps of a pair meet at unbounded named barriers, so their bounded waits (always on the same
+    // mbarrier) give up only on their own cycle limit: they watch a flag that nothing sets and raise the CTA's
+    volatile int* const own_limit_only = abort_flag + 1;
     bool ok = true;
 
     for (int j = 0; j < T; ++j) {
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), abort_flag, p.status, 31));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
@@ -308,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
       m_run = m_new;
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), abort_flag, p.status, 32));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
         if (!ok) break;
       }
       tc_fence_after();
@@ -348,7 +352,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
       if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
     }
 
-    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), abort_flag, p.status, 33));
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
     sMax[h * 128 + row] = l_run;
     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");

@@ -71,8 +71,10 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {     /
 // Bounded wait.  Returns false if the wait was abandoned (own limit reached, or another thread of
 // the CTA already gave up); the caller then skips to the teardown.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at full clock
+// `abort_flag` is the flag the wait watches; `raise_flag`, if given, is the one it sets on expiry instead.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code, long long limit = kWaitLimitCycles) {
+                                          int* status, int code, long long limit = kWaitLimitCycles,
+                                          volatile int* raise_flag = nullptr) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
@@ -80,7 +82,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if ((it & 15) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > limit) {
-        *abort_flag = 1;
+        *(raise_flag ? raise_flag : abort_flag) = 1;
         atomicCAS(status, 0, code);
         return false;
       }
