@@ -186,6 +186,30 @@ static HostPipe* host_pipe(size_t n_events) {
   return &hp;
 }
 
+// How many heads one pipeline stage of mxattn_forward_host takes.  A stage is one attention launch of
+// g * ceil(ceil(Nq/128)/2) CTAs on an n_sm-SM device: a partially filled last wave costs as much as a full
+// one (hunyuan: 466 CTAs per head = 3.15 waves on 148 SMs, 27 % lost at g = 1), while a larger g exposes more of
+// the first stage's host-to-device copy and of the last stage's device-to-host copy.  The estimate below
+// (attention at ~1.6 PFLOP/s, copies at ~50 GB/s) only has to rank the candidates.
+static int heads_per_stage(size_t bh, int64_t Nq, int64_t Nkv, size_t in_bytes_per_head, size_t out_bytes_per_head) {
+  int dev = 0, n_sm = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (n_sm <= 0) n_sm = 148;
+  const double ctas = (double)(((Nq + kTile - 1) / kTile + 1) / 2);
+  const double t_head = 4.0 * (double)Nq * (double)Nkv * kHeadDim / 1.6e15;
+  const double t_in = (double)in_bytes_per_head / 50e9, t_out = (double)out_bytes_per_head / 50e9;
+  int best = 1;
+  double best_t = 1e300;
+  for (int g = 1; g <= 8 && (size_t)g <= bh; ++g) {
+    if (g > 1 && bh / g < 3) break;                 // keep at least three stages to overlap
+    const double waves = g * ctas / n_sm;
+    const double eff = waves / (double)(int64_t)(waves + 0.999999);
+    const double t = (double)bh * t_head / eff + g * (t_in + t_out);
+    if (t < best_t * 0.995) { best_t = t; best = g; }
+  }
+  return best;
+}
+
 extern "C" size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags) {
   WorkspaceLayout w;
   if (!carve(1, 1, Nq, Nkv, d, &w) || B <= 0 || H <= 0) return 0;     // one workspace slice per head
@@ -215,43 +239,45 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   uint8_t* dv = dk + align_up(bh * kh, 256);
   uint8_t* dout = dv + align_up(bh * kh, 256);
   uint8_t* ws = dout + align_up(bh * oh, 256);
-  HostPipe* hp = host_pipe(2 * bh + 2);
+  const int g = heads_per_stage(bh, Nq, Nkv, qh + 2 * kh, oh);
+  const size_t stages = (bh + g - 1) / g;
+  HostPipe* hp = host_pipe(2 * stages + 2);
   if (!hp) return MXATTN_ECUDA;
   cudaEvent_t* ev = hp->ev.data();
   bool fail = false;
   auto ck = [&](cudaError_t e) { if (e != cudaSuccess) fail = true; };
-  ck(cudaEventRecord(ev[2 * bh], stream));                       // work already queued on the caller's stream comes first
-  ck(cudaStreamWaitEvent(hp->in, ev[2 * bh], 0));
+  ck(cudaEventRecord(ev[2 * stages], stream));                   // work already queued on the caller's stream comes first
+  ck(cudaStreamWaitEvent(hp->in, ev[2 * stages], 0));
   int rc = MXATTN_OK;
-  for (size_t i = 0; i < bh && !fail && rc == MXATTN_OK; ++i) {
-    const char* qs = static_cast<const char*>(q_host) + i * qh;
-    const char* ks = static_cast<const char*>(k_host) + i * kh;
-    const char* vs = static_cast<const char*>(v_host) + i * kh;
-    ck(cudaMemcpyAsync(dq + i * qh, qs, qh, cudaMemcpyHostToDevice, hp->in));
-    ck(cudaMemcpyAsync(dk + i * kh, ks, kh, cudaMemcpyHostToDevice, hp->in));
-    ck(cudaMemcpyAsync(dv + i * kh, vs, kh, cudaMemcpyHostToDevice, hp->in));
-    ck(cudaEventRecord(ev[2 * i], hp->in));
-    ck(cudaStreamWaitEvent(stream, ev[2 * i], 0));
-    rc = forward_ws(dq + i * qh, dk + i * kh, dv + i * kh, dout + i * oh, 1, 1, Nq, Nkv, d, softmax_scale, flags,
-                    ws + i * w.total, w.total, stream);
-    ck(cudaEventRecord(ev[2 * i + 1], stream));
-    ck(cudaStreamWaitEvent(hp->out, ev[2 * i + 1], 0));
-    ck(cudaMemcpyAsync(static_cast<char*>(o_host) + i * oh, dout + i * oh, oh, cudaMemcpyDeviceToHost, hp->out));
+  for (size_t st = 0; st < stages && !fail && rc == MXATTN_OK; ++st) {
+    const size_t i = st * g;                                     // first head of the stage; heads are contiguous in memory
+    const size_t n = (bh - i < (size_t)g) ? bh - i : (size_t)g;
+    ck(cudaMemcpyAsync(dq + i * qh, static_cast<const char*>(q_host) + i * qh, n * qh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaMemcpyAsync(dk + i * kh, static_cast<const char*>(k_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaMemcpyAsync(dv + i * kh, static_cast<const char*>(v_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
+    ck(cudaEventRecord(ev[2 * st], hp->in));
+    ck(cudaStreamWaitEvent(stream, ev[2 * st], 0));
+    // the stage's workspace starts at its first head's slice (n slices are at least as large as one workspace for n heads)
+    rc = forward_ws(dq + i * qh, dk + i * kh, dv + i * kh, dout + i * oh, 1, (int)n, Nq, Nkv, d, softmax_scale, flags,
+                    ws + i * w.total, n * w.total, stream);
+    ck(cudaEventRecord(ev[2 * st + 1], stream));
+    ck(cudaStreamWaitEvent(hp->out, ev[2 * st + 1], 0));
+    ck(cudaMemcpyAsync(static_cast<char*>(o_host) + i * oh, dout + i * oh, n * oh, cudaMemcpyDeviceToHost, hp->out));
   }
-  ck(cudaEventRecord(ev[2 * bh + 1], hp->out));
-  ck(cudaStreamWaitEvent(stream, ev[2 * bh + 1], 0));
+  ck(cudaEventRecord(ev[2 * stages + 1], hp->out));
+  ck(cudaStreamWaitEvent(stream, ev[2 * stages + 1], 0));
   // everything enqueued so far must drain before returning, also on an error path
   ck(cudaStreamSynchronize(hp->in));
   ck(cudaStreamSynchronize(stream));
   ck(cudaStreamSynchronize(hp->out));
-  g_launches = 4 * (int)bh;
+  g_launches = 4 * (int)stages;
   if (rc != MXATTN_OK) return rc;
   if (fail) return MXATTN_ECUDA;
-  // one status word per head, at the start of each workspace slice
-  std::vector<int> st(bh, 0);
-  if (cudaMemcpy2D(st.data(), sizeof(int), ws, w.total, sizeof(int), bh, cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
-  for (size_t i = 0; i < bh; ++i)
-    if (st[i]) return MXATTN_ETIMEOUT;
+  // one status word per stage, at the start of its workspace slice
+  std::vector<int> stw(stages, 0);
+  if (cudaMemcpy2D(stw.data(), sizeof(int), ws, (size_t)g * w.total, sizeof(int), stages, cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  for (size_t i = 0; i < stages; ++i)
+    if (stw[i]) return MXATTN_ETIMEOUT;
   return MXATTN_OK;
 }
 
