@@ -266,7 +266,11 @@ quantize_axis1_rot_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ co
 }
 
 // ------------------------------------------------------------------------------------------
-// Axis 0.  grid = (ceil(cols/128), ceil(rows/128), batch); 256 threads.
+// Axis 0.  256 threads; a CTA stages a 32 KiB slab of the input in shared memory:
+//   tile layout:  128 tokens x 128 columns -> one 8.5 KiB tile image, written contiguously;
+//                 grid = (1, ceil(rows/128), batch)
+//   canonical:    256 tokens x 64 columns, so that every column leaves as ONE 128-byte segment of codes
+//                 (and 8 scale bytes) instead of two 64-byte ones; grid = (ceil(cols/64), ceil(rows_pad/256), batch)
 constexpr int kVThreads = 256;
 
 template <bool kTileLayout>
@@ -274,21 +278,28 @@ __global__ void __launch_bounds__(kVThreads)
 quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t rows, int64_t cols, int64_t rows_pad,
                       uint32_t rule) {
-  __shared__ __align__(16) uint16_t s_in[kTile][kTile];           // [token][column] raw bf16
-  __shared__ __align__(16) uint8_t s_codes[kTileCodeBytes];       // [column][64 B] (swizzled if tile layout)
+  constexpr int kTok = kTileLayout ? 128 : 256;                   // tokens per slab
+  constexpr int kCol = kTileLayout ? 128 : 64;                    // columns per slab
+  constexpr int kColBytes = kTok / 2;                             // code bytes per column of the slab
+  constexpr int kColBlocks = kTok / kBlock;                       // blocks (scale bytes) per column of the slab
+  __shared__ __align__(16) uint16_t s_in[kTok][kCol];             // [token][column] raw bf16
+  __shared__ __align__(16) uint8_t s_codes[kTileCodeBytes];       // [column][kColBytes], 16-byte chunks swizzled
   __shared__ __align__(16) uint8_t s_scales[kTileScaleBytes];
 
   const int tid = threadIdx.x;
-  const int64_t col0 = (int64_t)blockIdx.x * kTile;
-  const int64_t row0 = (int64_t)blockIdx.y * kTile;
+  const int64_t col0 = (int64_t)blockIdx.x * kCol;
+  const int64_t row0 = (int64_t)blockIdx.y * kTok;
   const int64_t b = blockIdx.z;
   const uint16_t* src = in + b * rows * cols;
+  // staging offset of the 16-byte chunk c of column n: the tile image's own swizzle, or (canonical) the
+  // chunk index XORed with the column pair so that the 8 threads of a store phase hit 8 different bank groups
+  auto code_off = [](int n, int c) { return kTileLayout ? tile_code_offset(n, c) : n * kColBytes + ((c ^ ((n >> 1) & 7)) << 4); };
 
-  // phase 1: 128 x 128 bf16 slab -> shared, 16 B per thread per step, zero beyond the edges
+  // phase 1: slab -> shared, 16 B per thread per step, zero beyond the edges
 #pragma unroll
-  for (int k = 0; k < (kTile * kTile / 8) / kVThreads; ++k) {
-    const int chunk = k * kVThreads + tid;      // 16 chunks per token row
-    const int t = chunk >> 4, cc = (chunk & 15) << 3;
+  for (int k = 0; k < (kTok * kCol / 8) / kVThreads; ++k) {
+    const int chunk = k * kVThreads + tid;
+    const int t = chunk / (kCol / 8), cc = (chunk % (kCol / 8)) << 3;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (row0 + t < rows && col0 + cc < cols)
       v = __ldg(reinterpret_cast<const uint4*>(src + (row0 + t) * cols + col0 + cc));
@@ -299,13 +310,13 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
   // phase 2: thread -> (column pair 2np, 2np+1; token block c).  One 32-bit shared load brings both
   // columns of a token, so the packed maximum and the two conversions share the 32 loads.
   {
-    const int np = tid & 63, c = tid >> 6;
+    const int np = tid % (kCol / 2), c = tid / (kCol / 2);
     const uint32_t* s32 = reinterpret_cast<const uint32_t*>(&s_in[0][0]);
     uint32_t w[32];
     uint32_t m2 = 0;
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-      w[i] = s32[(c * 32 + i) * (kTile / 2) + np];
+      w[i] = s32[(c * 32 + i) * (kCol / 2) + np];
       m2 = __vmaxu2(m2, w[i] & 0x7FFF7FFFu);
     }
 #pragma unroll
@@ -322,14 +333,13 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
         for (int i = 0; i < 8; ++i) f[i] = (side ? bf16hi(w[8 * q + i]) : bf16lo(w[8 * q + i])) * inv;
         o[q] = pack_e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
       }
-      const int coff = kTileLayout ? tile_code_offset(n, c) : (n * 64 + c * 16);
-      *reinterpret_cast<uint4*>(&s_codes[coff]) = make_uint4(o[0], o[1], o[2], o[3]);
-      s_scales[kTileLayout ? tile_scale_offset(n, c) : (n * 4 + c)] = (uint8_t)(e + 127);
+      *reinterpret_cast<uint4*>(&s_codes[code_off(n, c)]) = make_uint4(o[0], o[1], o[2], o[3]);
+      s_scales[kTileLayout ? tile_scale_offset(n, c) : (n * kColBlocks + c)] = (uint8_t)(e + 127);
     }
   }
   __syncthreads();
 
-  // phase 3: staged tile -> global
+  // phase 3: staged slab -> global
   if (kTileLayout) {
     const int64_t tile = b * gridDim.y + blockIdx.y;            // cols == 128: one column tile
     uint4* dst = reinterpret_cast<uint4*>(codes + tile * kTileCodeBytes);
@@ -340,20 +350,25 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
       reinterpret_cast<uint4*>(scales + tile * kTileScaleBytes)[tid] =
           reinterpret_cast<const uint4*>(s_scales)[tid];
   } else {
-    // codes [cols, rows_pad/2]: column n owns 64 contiguous bytes of this token tile
+    // codes [cols, rows_pad/2]: column n owns kColBytes contiguous bytes of this slab (the second 128 tokens
+    // only if they are inside rows_pad, which is a multiple of 128, not of 256)
     uint8_t* cdst = codes + b * cols * (rows_pad / 2);
     uint8_t* sdst = scales + b * cols * (rows_pad / 32);
+    const bool second = row0 + 128 < rows_pad;
 #pragma unroll
     for (int k = 0; k < kTileCodeBytes / 16 / kVThreads; ++k) {
       const int chunk = k * kVThreads + tid;
-      const int n = chunk >> 2, q = chunk & 3;
-      if (col0 + n < cols)
+      const int n = chunk / (kColBytes / 16), q = chunk % (kColBytes / 16);
+      if (col0 + n < cols && (q < 4 || second))
         *reinterpret_cast<uint4*>(cdst + (col0 + n) * (rows_pad / 2) + row0 / 2 + q * 16) =
-            reinterpret_cast<const uint4*>(s_codes)[chunk];
+            *reinterpret_cast<const uint4*>(&s_codes[code_off(n, q)]);
     }
-    if (tid < kTile && col0 + tid < cols)
-      *reinterpret_cast<uint32_t*>(sdst + (col0 + tid) * (rows_pad / 32) + row0 / 32) =
-          reinterpret_cast<const uint32_t*>(s_scales)[tid];
+    if (tid < 2 * kCol) {
+      const int n = tid >> 1, half = tid & 1;
+      if (col0 + n < cols && (half == 0 || second))
+        *reinterpret_cast<uint32_t*>(sdst + (col0 + n) * (rows_pad / 32) + row0 / 32 + 4 * half) =
+            reinterpret_cast<const uint32_t*>(s_scales)[n * 2 + half];
+    }
   }
 }
 
@@ -404,10 +419,11 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
             (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
     }
   } else {
-    const int64_t ct = (cols + kTile - 1) / kTile, rt = rows_pad / kTile;
-    if (rt > 65535 || batch > 65535) return MXATTN_EUNSUPPORTED;
+    const bool tile = (layout == MXATTN_LAYOUT_TILE);
+    const int64_t ct = tile ? 1 : (cols + 63) / 64, rt = tile ? rows_pad / kTile : (rows_pad + 255) / 256;
+    if (ct > 0x7FFFFFFF || rt > 65535 || batch > 65535) return MXATTN_EUNSUPPORTED;
     dim3 grid((unsigned)ct, (unsigned)rt, (unsigned)batch);
-    if (layout == MXATTN_LAYOUT_TILE)
+    if (tile)
       quantize_axis0_kernel<true><<<grid, kVThreads, 0, stream>>>(
           (const uint16_t*)in, (uint8_t*)codes, (uint8_t*)scales, rows, cols, rows_pad, rule);
     else
