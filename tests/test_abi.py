@@ -41,3 +41,23 @@ def test_argument_errors_need_no_device():
     mx.set_workspace(None)
     assert L.mxattn_forward(16, 16, 16, 16, 1, 2, 128, 128, 128, 0.1, 3, None) == -4      # no workspace
     assert mx.strerror(-6).startswith("device-side")
+
+
+def test_argument_errors_of_the_diagnostic_entry_points():
+    import paper_2607_24377_b200 as mx
+    L = mx.lib()
+    big = 1 << 40
+    # row-sum diagnostic: flags other than UOS / HADAMARD, head dimension, alignment, workspace
+    assert L.mxattn_rowsum_diagnostic(16, 16, 16, 1, 1, 128, 128, 128, 0.1, 2, 16, big, None) == -1     # PNQ is no flag of it
+    assert L.mxattn_rowsum_diagnostic(None, 16, 16, 1, 1, 128, 128, 128, 0.1, 1, 16, big, None) == -1
+    assert L.mxattn_rowsum_diagnostic(16, 16, 16, 1, 1, 128, 128, 64, 0.1, 1, 16, big, None) == -2
+    assert L.mxattn_rowsum_diagnostic(16, 24, 16, 1, 1, 128, 128, 128, 0.1, 1, 16, big, None) == -3
+    assert L.mxattn_rowsum_diagnostic(16, 16, 16, 1, 1, 128, 128, 128, 0.1, 1, 16, 1024, None) == -4
+    assert L.mxattn_rowsum_diagnostic(16, 16, 16, 1, 1, 128, 128, 128, 0.0, 1, 16, big, None) == -1
+    # debug dump: needs the dump buffer, the fp32 output flag, a buffer of the stated size, a small problem
+    assert mx.forward_debug_dump_bytes(1, 2, 1024, 1024, 128) == 2 * 8 * 8 * 9216 + 2 * 8 * 128 * 4
+    assert mx.forward_debug_dump_bytes(1, 2, 1024, 1024, 64) == 0
+    assert L.mxattn_forward_debug_dump(16, 16, 16, 16, 1, 2, 1024, 1024, 128, 0.1, 7, 16, big, None, big, None) == -1
+    assert L.mxattn_forward_debug_dump(16, 16, 16, 16, 1, 2, 1024, 1024, 128, 0.1, 3, 16, big, 16, big, None) == -1   # bf16 output
+    assert L.mxattn_forward_debug_dump(16, 16, 16, 16, 1, 2, 1024, 1024, 128, 0.1, 7, 16, big, 16, 1024, None) == -4
+    assert L.mxattn_forward_debug_dump(16, 16, 16, 16, 1, 40, 75600, 75600, 128, 0.1, 7, 16, big, 16, big, None) == -2
