@@ -126,7 +126,7 @@ def run_reference(args, cfg):
         return
     import numpy  # noqa: F401  (BLAS threads are whatever the environment gives the oracle)
     heads = [0]
-    rows = 16 if cfg.Nkv > 20000 else 64
+    rows = min(cfg.Nq, 256 if cfg.Nkv > 20000 else 512)     # a few seconds per step
     vals = []
     for i in range(args.warmup + args.steps):
         tf, dt, desc = oracle_sample(cfg, heads, rows)
@@ -336,7 +336,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         heads = [0, 1] if Nkv <= 20000 else [0]
-        rows = 64 if Nkv <= 20000 else 32
+        rows = min(cfg.Nq, 2048)                   # about 10-20 s of oracle time at the wan22 size
         tf, dt, desc = oracle_sample(cfg, heads, rows)
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
                         "seconds": dt}
