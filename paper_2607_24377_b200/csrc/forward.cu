@@ -68,13 +68,13 @@ constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
 constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
 constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
-constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2 + 2;  // Q, K/V full+empty, S_full[2], S_free, P_full[2], O_done[2]
+constexpr int kNumBars = 1 + 2 * kStages + 2 + 1 + 2 + 2;  // Q, K/V stage full+empty, S_full[2], S_free, P_full[2], O_done[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
 constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
 
-enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages, BAR_VFULL = BAR_KEMPTY + kStages,
-           BAR_VEMPTY = BAR_VFULL + kStages, BAR_SFULL = BAR_VEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
+enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages,     // one full / empty pair per K/V stage
+           BAR_SFULL = BAR_KEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
            BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2 };
 
 // tensor-memory columns
@@ -116,7 +116,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     mbar_init(bar(BAR_Q), 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(BAR_KFULL + s), 1); mbar_init(bar(BAR_KEMPTY + s), 1);
-      mbar_init(bar(BAR_VFULL + s), 1); mbar_init(bar(BAR_VEMPTY + s), 1);
     }
     mbar_init(bar(BAR_SFULL + 0), 1); mbar_init(bar(BAR_SFULL + 1), 1);
     mbar_init(bar(BAR_SFREE), 4 * kSplit);                  // one arrival per softmax warp of the draining group
@@ -162,14 +161,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         const uint32_t ph = (uint32_t)((j / kStages) & 1);
         if (j >= kStages) ok = mbar_wait(bar(BAR_KEMPTY + s), ph ^ 1u, abort_flag, p.status, 11);
         if (!ok) break;
-        mbar_expect_tx(bar(BAR_KFULL + s), kTileCodeBytes + kTileScaleBytes);
+        // K-hat_j and V-hat_j travel together: one full / one empty barrier per stage (the issuer thread's time
+        // per tile is what bounds the kernel, and every wait or commit it does not need shortens it)
+        mbar_expect_tx(bar(BAR_KFULL + s), 2 * (kTileCodeBytes + kTileScaleBytes));
         bulk_g2s(sbase + kOffK + s * kTileCodeBytes, p.k_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
         bulk_g2s(sbase + kOffSFK + s * kTileScaleBytes, p.k_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
-        if (j >= kStages) ok = mbar_wait(bar(BAR_VEMPTY + s), ph ^ 1u, abort_flag, p.status, 12);
-        if (!ok) { issued = j + 1; break; }   // K(j) is in flight, V(j) is not
-        mbar_expect_tx(bar(BAR_VFULL + s), kTileCodeBytes + kTileScaleBytes);
-        bulk_g2s(sbase + kOffV + s * kVStageBytes, p.v_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_VFULL + s));
-        bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_VFULL + s));
+        bulk_g2s(sbase + kOffV + s * kVStageBytes, p.v_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
+        bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
         issued = j + 1;
       }
       if (!ok || *abort_flag) {
@@ -179,7 +177,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
           const uint32_t ph = (uint32_t)((j / kStages) & 1);
           const long long t0 = clock64();
           while (!mbar_try(bar(BAR_KFULL + s), ph) && clock64() - t0 < 200000000LL) {}
-          while (!mbar_try(bar(BAR_VFULL + s), ph) && clock64() - t0 < 200000000LL) {}
         }
         const long long t0 = clock64();
         while (!mbar_try(bar(BAR_Q), 0) && clock64() - t0 < 200000000LL) {}
@@ -215,11 +212,19 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         tc_mma(d, desc(a + 2), desc(b + 2), make_idesc(kNV, 1), sfa, sfb, 1u);
         tc_commit(bar(BAR_ODONE + t));
       };
-      auto wait_k = [&](int j) {
+      // K-hat_j and V-hat_j have landed (and, unless `first`, the score buffer is free): one fence, then the scale
+      // atoms of both go to tensor memory -- V's two tiles ahead of its GEMM, which keeps that copy out of the
+      // path from "P is ready" to "GEMM 2 issued" (slot j & 1 was last read by the GEMMs of tile j - 2, issued before)
+      auto wait_kv = [&](int j, bool first) {
         const int s = j % kStages;
         if (!mbar_wait(bar(BAR_KFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 22)) return false;
+        if (!first) {
+          if (!mbar_wait(bar(BAR_SFREE), sfree_n & 1u, abort_flag, p.status, 23)) return false;
+          ++sfree_n;
+        }
         tc_fence_after();
         tc_cp_sf(tmem + kColSFK + 4 * (j & 1), sbase + kOffSFK + s * kTileScaleBytes);
+        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
         return true;
       };
       auto wait_sfree = [&]() {
@@ -236,37 +241,32 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
       }
       // prologue: S(0,0), S(1,0), S(0,1)
-      ok = ok && wait_k(0);
+      ok = ok && wait_kv(0, true);
       if (ok) gemm1(0, 0);
       ok = ok && wait_sfree();
-      if (ok) { gemm1(1, 0); tc_commit(bar(BAR_KEMPTY + 0)); }
+      if (ok) gemm1(1, 0);
       if (T > 1) {
-        ok = ok && wait_k(1);
-        ok = ok && wait_sfree();
+        ok = ok && wait_kv(1, false);
         if (ok) gemm1(0, 1);
       }
       for (int j = 0; j < T && ok; ++j) {
         const int s = j % kStages;
-        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);
-        ok = ok && mbar_wait(bar(BAR_VFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 25);
+        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);     // V_j arrived with K_j
         if (!ok) break;
         tc_fence_after();
-        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
         gemm2(0, j);
         if (j + 1 < T) {
           ok = wait_sfree();
           if (!ok) break;
           gemm1(1, j + 1);
-          tc_commit(bar(BAR_KEMPTY + (j + 1) % kStages));
         }
         ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
         if (!ok) break;
         tc_fence_after();
         gemm2(1, j);
-        tc_commit(bar(BAR_VEMPTY + s));
+        tc_commit(bar(BAR_KEMPTY + s));            // the last reader of stage s: K_j and V_j may be overwritten
         if (j + 2 < T) {
-          ok = wait_k(j + 2);
-          ok = ok && wait_sfree();
+          ok = wait_kv(j + 2, false);
           if (!ok) break;
           gemm1(0, j + 2);
         }
