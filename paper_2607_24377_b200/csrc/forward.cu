@@ -388,12 +388,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         if (h == 0) reinterpret_cast<float*>(dump_tile + kTileCodeBytes + kTileScaleBytes)[row] = m_new * p.softmax_scale;   // the kernel keeps m in unscaled score units
       }
       float l_tile = 0.0f;
+      const uint64_t cc2 = dup2(c);
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
         if (kResc) alpha = ex2((m_old - m_new) * c);
 #pragma unroll
         for (int b = 0; b < kBlocksPerThread; ++b) {
-          const float nb = nbs[b];
+          const uint64_t nb2 = dup2(nbs[b]);
           uint4 w;
           float sx = 0.0f;
 #pragma unroll
@@ -403,7 +404,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
             if (kResc) TMEM_LD8(t_oc, oc);
             float x[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = ex2(fmaf(__uint_as_float(sr[32 * b + 8 * g + i]), c, nb));
+            for (int i = 0; i < 8; i += 2) {           // x = exp2(s * c + nb), two elements per multiply-add
+              fma2(sr[32 * b + 8 * g + i], sr[32 * b + 8 * g + i + 1], cc2, nb2, x[i], x[i + 1]);
+              x[i] = ex2(x[i]);
+              x[i + 1] = ex2(x[i + 1]);
+            }
             const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
             if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
             if (!kPnq) sx += ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));

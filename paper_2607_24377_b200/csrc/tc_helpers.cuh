@@ -29,6 +29,19 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+// Two fused multiply-adds in one instruction (packed fp32x2): (a0, a1) * cc + dd with cc = (c, c), dd = (d, d);
+// each half is an IEEE fp32 fma, bit-identical to fmaf.
+__device__ __forceinline__ uint64_t dup2(float v) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(r) : "f"(v));
+  return r;
+}
+__device__ __forceinline__ void fma2(uint32_t a0_bits, uint32_t a1_bits, uint64_t cc, uint64_t dd, float& r0, float& r1) {
+  uint64_t ab, r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ab) : "r"(a0_bits), "r"(a1_bits));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(ab), "l"(cc), "l"(dd));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(r));
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
