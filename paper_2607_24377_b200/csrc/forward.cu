@@ -249,6 +249,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         ok = ok && wait_kv(1, false);
         if (ok) gemm1(0, 1);
       }
+      // unrolled by the number of stages: stage indices, parities and descriptor offsets become constants, and the
+      // thread's scalar instructions between its tcgen05 instructions are part of the kernel's critical path
+#pragma unroll 4
       for (int j = 0; j < T && ok; ++j) {
         const int s = j % kStages;
         ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);     // V_j arrived with K_j
