@@ -32,9 +32,9 @@ NOMINAL_FP4_TFLOPS = 9000.0      # dense FP4, nominal
 FP4_OVER_BF16 = 4.0              # nominal ratio of dense FP4 to dense bf16 tensor throughput
 QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0
 # DRAM bytes of one attention launch, from the ncu capture of the same kernel on sweep16384
-# (256.7 MB, profiles/attention_kernel_sweep16384.txt) scaled by tokens x heads (traffic follows the
+# (253.0 MB, profiles/attention_kernel_sweep16384.txt) scaled by tokens x heads (traffic follows the
 # operand bytes, not the flops).
-ATTN_TRAFFIC_PER_TOKEN_HEAD = 256.7e6 / (16384 * 40)
+ATTN_TRAFFIC_PER_TOKEN_HEAD = 253.0e6 / (16384 * 40)
 
 
 def load_peaks():
