@@ -336,14 +336,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       float own_max = bmax[0];
 #pragma unroll
       for (int b = 1; b < kBlocksPerThread; ++b) own_max = fmaxf(own_max, bmax[b]);
-      // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t
-      // or rescales O_t; probe that barrier early so its latency overlaps other work
-      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
       // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
       const uint32_t par = (uint32_t)(j & 1) * 2048u;
       sts32f(aMaxOwn + par, own_max);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
-      const float m_new = max3(m_run, own_max, lds32f(aMaxPartner + par));   // line 10
+      const float partner_max = lds32f(aMaxPartner + par);
+      // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t or rescales
+      // O_t; the probe of that barrier is issued while the partner's maximum is on its way
+      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
+      const float m_new = max3(m_run, own_max, partner_max);   // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
