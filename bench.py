@@ -336,7 +336,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         heads = [0, 1] if Nkv <= 20000 else [0]
-        rows = min(cfg.Nq, 2048)                   # about 10-20 s of oracle time at the wan22 size
+        rows = min(cfg.Nq, 6144)                   # about 10-15 s of oracle time at the wan22 size on a 16-core host
         tf, dt, desc = oracle_sample(cfg, heads, rows)
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
                         "seconds": dt}
