@@ -6,8 +6,12 @@
 //               (warps 0-3 take columns 0-63, warps 4-7 columns 64-127; warp w works on the
 //               tensor-memory lanes 32*(w%4) .. +31, i.e. rows 32*(w%4) .. +31 of the tile)
 //   warps 8-15  softmax group 1 (query tile 1), same split
-//   warp  16    producer: bulk async copies (TMA unit) of K-hat / V-hat tile images + scale atoms
-//   warp  17    MMA issuer: block-scaled FP4 tcgen05.mma (kind::mxf4, E8M0 scales), one thread
+//   warp  16    producer: bulk async copies (TMA unit) of K-hat / V-hat tile images + scale atoms, four
+//               stages; the K and V images of a tile complete one mbarrier
+//   warp  17    MMA issuer: block-scaled FP4 tcgen05.mma (kind::mxf4, E8M0 scales), one thread.  What this
+//               thread does per tile (5 waits, 4 scale-atom copies, 8 MMAs, 5 commits and the scalar
+//               instructions between them) is on the kernel's critical path, so its loop is kept as short
+//               as the dependencies allow and is unrolled by the number of stages.
 //
 // Both GEMMs are dense FP4 contractions with fp32 accumulators in tensor memory:
 //   GEMM 1  S   = Q-hat_t K-hat_j^T              (M=128, N=128, K=128 as two K=64 instructions)
@@ -28,8 +32,8 @@
 //     codes = RNE-to-E2M1(x), 16 bytes, written into the K-major, 64B-swizzled A-operand tile
 //   and its two scale bytes into the scale-factor atom.  The difference (bmax_b - m_new) is formed
 //   exactly first, so the block holding the row maximum has d = 0 and gets e = -2 under both rules,
-//   the scale the paper's Appendix J derives; the elements take one fused multiply-add and one
-//   ex2.approx each.
+//   the scale the paper's Appendix J derives; the elements take one fused multiply-add (issued two at a
+//   time as a packed fp32x2 instruction) and one ex2.approx each.
 //   If a row maximum of the warp moved, the thread rescales its 64 accumulator columns in tensor
 //   memory by alpha = exp(m - m_new) (line 15); those tensor-memory round trips are interleaved with
 //   the exponentials (the loop body exists in two straight-line versions).
@@ -38,7 +42,7 @@
 // to registers at once, so the buffer is free again long before the other group needs it),
 // O_0 [128,272), O_1 [272,416), scale factors from 416.
 //
-// Every wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
+// Every mbarrier wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
 #include <type_traits>
 
 #include "common.cuh"
