@@ -35,9 +35,13 @@ static bool carve(int B, int H, int64_t Nq, int64_t Nkv, int d, WorkspaceLayout*
   return true;
 }
 
+// `qstream` / `qdone`: if given, the three quantize launches go to `qstream`, `qdone` is recorded behind them and
+// the attention launch on `stream` waits for it (the host pipeline uses this to quantize the next stage's
+// operands while the current stage's attention kernel drains).
 static int forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq,
                       int64_t Nkv, int d, float softmax_scale, unsigned flags, void* workspace,
-                      size_t workspace_bytes, cudaStream_t stream, void* dump = nullptr) {
+                      size_t workspace_bytes, cudaStream_t stream, void* dump = nullptr,
+                      cudaStream_t qstream = nullptr, cudaEvent_t qdone = nullptr) {
   if (!q || !k || !v || !o) return MXATTN_EINVAL;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
   if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32 | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
@@ -53,12 +57,16 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
   const int mode = (flags & MXATTN_FLAG_UOS) ? MXATTN_MODE_UOS : MXATTN_MODE_OCP;
   const int qk_mode = mode | ((flags & MXATTN_FLAG_HADAMARD) ? MXATTN_MODE_HADAMARD : 0);   // Algorithm 2 lines 1-2
   const int64_t bh = (int64_t)B * H;
-  if (cudaMemsetAsync(ws + w.status, 0, 16, stream) != cudaSuccess) return MXATTN_ECUDA;
+  cudaStream_t qs = qstream ? qstream : stream;
+  if (cudaMemsetAsync(ws + w.status, 0, 16, qs) != cudaSuccess) return MXATTN_ECUDA;
   int rc;
   // Algorithm 2 lines 3-5: Q-hat, K-hat (blocks along d), V-hat (blocks along tokens)
-  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
-  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, stream))) return rc;
-  if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, stream))) return rc;
+  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+  if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+  if (qstream) {
+    if (cudaEventRecord(qdone, qstream) != cudaSuccess || cudaStreamWaitEvent(stream, qdone, 0) != cudaSuccess) return MXATTN_ECUDA;
+  }
   // lines 6-19
   return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
                         ws + w.v_scales, o, B, H, Nq, Nkv, softmax_scale, flags,
@@ -167,7 +175,7 @@ extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_sc
 // kernels of head h (PCIe is full duplex).  The two helper streams and the events are created on
 // first use, once per device, and kept for the life of the process; no device memory is allocated.
 struct HostPipe {
-  cudaStream_t in = nullptr, out = nullptr;
+  cudaStream_t in = nullptr, quant = nullptr, out = nullptr;
   std::vector<cudaEvent_t> ev;
 };
 static HostPipe g_pipe[64];
@@ -178,6 +186,7 @@ static HostPipe* host_pipe(size_t n_events) {
   HostPipe& hp = g_pipe[dev];
   if (!hp.in && cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   if (!hp.out && cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (!hp.quant && cudaStreamCreateWithFlags(&hp.quant, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   while (hp.ev.size() < n_events) {
     cudaEvent_t e;
     if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
@@ -241,13 +250,13 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   uint8_t* ws = dout + align_up(bh * oh, 256);
   const int g = heads_per_stage(bh, Nq, Nkv, qh + 2 * kh, oh);
   const size_t stages = (bh + g - 1) / g;
-  HostPipe* hp = host_pipe(2 * stages + 2);
+  HostPipe* hp = host_pipe(3 * stages + 2);
   if (!hp) return MXATTN_ECUDA;
   cudaEvent_t* ev = hp->ev.data();
   bool fail = false;
   auto ck = [&](cudaError_t e) { if (e != cudaSuccess) fail = true; };
-  ck(cudaEventRecord(ev[2 * stages], stream));                   // work already queued on the caller's stream comes first
-  ck(cudaStreamWaitEvent(hp->in, ev[2 * stages], 0));
+  ck(cudaEventRecord(ev[3 * stages], stream));                   // work already queued on the caller's stream comes first
+  ck(cudaStreamWaitEvent(hp->in, ev[3 * stages], 0));
   int rc = MXATTN_OK;
   for (size_t st = 0; st < stages && !fail && rc == MXATTN_OK; ++st) {
     const size_t i = st * g;                                     // first head of the stage; heads are contiguous in memory
@@ -255,19 +264,22 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
     ck(cudaMemcpyAsync(dq + i * qh, static_cast<const char*>(q_host) + i * qh, n * qh, cudaMemcpyHostToDevice, hp->in));
     ck(cudaMemcpyAsync(dk + i * kh, static_cast<const char*>(k_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
     ck(cudaMemcpyAsync(dv + i * kh, static_cast<const char*>(v_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
-    ck(cudaEventRecord(ev[2 * st], hp->in));
-    ck(cudaStreamWaitEvent(stream, ev[2 * st], 0));
-    // the stage's workspace starts at its first head's slice (n slices are at least as large as one workspace for n heads)
+    ck(cudaEventRecord(ev[3 * st], hp->in));
+    ck(cudaStreamWaitEvent(hp->quant, ev[3 * st], 0));
+    // the stage's workspace starts at its first head's slice (n slices are at least as large as one workspace for
+    // n heads); its operands are quantized on a stream of their own, behind the copies and ahead of the attention
+    // launch, so that they fill the SMs the previous stage's attention kernel frees as it drains
     rc = forward_ws(dq + i * qh, dk + i * kh, dv + i * kh, dout + i * oh, 1, (int)n, Nq, Nkv, d, softmax_scale, flags,
-                    ws + i * w.total, n * w.total, stream);
-    ck(cudaEventRecord(ev[2 * st + 1], stream));
-    ck(cudaStreamWaitEvent(hp->out, ev[2 * st + 1], 0));
+                    ws + i * w.total, n * w.total, stream, nullptr, hp->quant, ev[3 * st + 1]);
+    ck(cudaEventRecord(ev[3 * st + 2], stream));
+    ck(cudaStreamWaitEvent(hp->out, ev[3 * st + 2], 0));
     ck(cudaMemcpyAsync(static_cast<char*>(o_host) + i * oh, dout + i * oh, n * oh, cudaMemcpyDeviceToHost, hp->out));
   }
-  ck(cudaEventRecord(ev[2 * stages + 1], hp->out));
-  ck(cudaStreamWaitEvent(stream, ev[2 * stages + 1], 0));
+  ck(cudaEventRecord(ev[3 * stages + 1], hp->out));
+  ck(cudaStreamWaitEvent(stream, ev[3 * stages + 1], 0));
   // everything enqueued so far must drain before returning, also on an error path
   ck(cudaStreamSynchronize(hp->in));
+  ck(cudaStreamSynchronize(hp->quant));
   ck(cudaStreamSynchronize(stream));
   ck(cudaStreamSynchronize(hp->out));
   g_launches = 4 * (int)stages;
