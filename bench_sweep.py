@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Sweep report (BASELINE configs[1] and configs[4]); prints one JSON document.
+"""Sweep report (the outlier configuration and the N sweep of the benchmark definition); prints one JSON document.
 
     python bench_sweep.py [--quick]
 

@@ -62,13 +62,13 @@ class AttnConfig:
 
 
 CONFIGS = {
-    # BASELINE configs[0..3]
+    # the four named configurations of the benchmark definition
     "tiny": AttnConfig("tiny", 1, 2, 1024, 1024, 0, "iid"),
     "outlier": AttnConfig("outlier", 1, 24, 8192, 8192, 1, "outlier"),
     "wan22": AttnConfig("wan22", 1, 40, 75600, 75600, 2, "wan"),
     "hunyuan": AttnConfig("hunyuan", 1, 24, 119056, 119056, 3, "hunyuan"),
 }
-for _n in (4096, 16384, 32768, 65536):  # BASELINE configs[4], the sweep
+for _n in (4096, 16384, 32768, 65536):  # the N sweep of the benchmark definition
     CONFIGS[f"sweep{_n}"] = AttnConfig(f"sweep{_n}", 1, 40, _n, _n, 100 + int(math.log2(_n)), "outlier")
 
 # Wan2.2 has separate cross-attention modules (paper Section 5.1): video queries against a short text
