@@ -470,6 +470,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         l = __uint_as_float(lr);
       }
       const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
+      const float inv_l = 1.0f / l;                // line 18 as one reciprocal and 64 multiplies per thread
       if (kDump && h == 0 && qtile < p.q_tiles)
         reinterpret_cast<float*>(p.dump + (int64_t)gridDim.x / p.q_pairs * p.q_tiles * T * kDumpTileBytes)
             [((int64_t)bh * p.q_tiles + qtile) * kTile + row] = l;
@@ -484,8 +485,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
             float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + obase + c0);
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-              dst[i] = make_float4(__uint_as_float(r32[4 * i]) / l, __uint_as_float(r32[4 * i + 1]) / l,
-                                   __uint_as_float(r32[4 * i + 2]) / l, __uint_as_float(r32[4 * i + 3]) / l);
+              dst[i] = make_float4(__uint_as_float(r32[4 * i]) * inv_l, __uint_as_float(r32[4 * i + 1]) * inv_l,
+                                   __uint_as_float(r32[4 * i + 2]) * inv_l, __uint_as_float(r32[4 * i + 3]) * inv_l);
           } else {
             uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + obase + c0);
 #pragma unroll
@@ -493,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
               uint32_t hh[4];
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
-                const float a = __uint_as_float(r32[8 * i + 2 * k]) / l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) / l;
+                const float a = __uint_as_float(r32[8 * i + 2 * k]) * inv_l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) * inv_l;
                 asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hh[k]) : "f"(b2), "f"(a));
               }
               dst[i] = make_uint4(hh[0], hh[1], hh[2], hh[3]);
