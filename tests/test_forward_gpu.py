@@ -104,9 +104,12 @@ def test_prequantized_entry_equals_full_forward():
     assert torch.equal(out, full)
 
 
-def test_host_buffer_entry_point():
+@pytest.mark.parametrize("B,H", [(1, 2), (1, 13), (2, 7)])
+def test_host_buffer_entry_point(B, H):
+    # 2 heads: one head per pipeline stage; 13 and 14 heads of a single query-tile pair: several heads per stage
+    # (a stage should fill the SMs), with a shorter last stage
     import paper_2607_24377_b200 as mx
-    cfg = si.custom_config("h", 1, 2, 256, 512, 81)
+    cfg = si.custom_config("h", B, H, 256, 512, 81)
     q, k, v = si.make_all(cfg)
     want = run_forward(cfg, q, k, v, True, True).cpu()
     hq, hk, hv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (q, k, v))
@@ -115,6 +118,9 @@ def test_host_buffer_entry_point():
     arena = torch.empty(mx.forward_host_arena_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, flags), dtype=torch.uint8, device="cuda")
     mx.forward_host(hq, hk, hv, ho, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, 128, cfg.softmax_scale, flags, arena)
     assert torch.equal(ho, want)
+    assert mx.last_launch_count() % 4 == 0 and mx.last_launch_count() <= 4 * B * H
+    if B * H >= 12:
+        assert mx.last_launch_count() < 4 * B * H          # heads were grouped into stages
 
 
 @pytest.mark.parametrize("recipe", ["iid", "outlier", "wan"])
