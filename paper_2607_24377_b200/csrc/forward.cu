@@ -62,24 +62,28 @@ constexpr int kVStageBytes = kNV * 64;           // 9216
 constexpr int kDumpTileBytes = kTileCodeBytes + kTileScaleBytes + kTile * 4;   // debug dump: codes, scale atom, m per row
 
 // shared memory map (byte offsets from a 1024-aligned base)
-constexpr int kOffQ = 0;                                   // 2 x 8192
-constexpr int kOffK = kOffQ + 2 * kTileCodeBytes;          // 4 x 8192
+constexpr int kOffQ = 0;                                   // 2 buffers x 2 tiles x 8192 (the second buffer: persistent variant)
+constexpr int kOffK = kOffQ + 4 * kTileCodeBytes;          // 4 x 8192
 constexpr int kOffV = kOffK + kStages * kTileCodeBytes;    // 4 x 9216
 constexpr int kOffP = kOffV + kStages * kVStageBytes;      // 2 x 8192
-constexpr int kOffSFQ = kOffP + 2 * kTileCodeBytes;        // 2 x 512
-constexpr int kOffSFK = kOffSFQ + 2 * kTileScaleBytes;     // 4 x 512
+constexpr int kOffSFQ = kOffP + 2 * kTileCodeBytes;        // 2 buffers x 2 x 512
+constexpr int kOffSFK = kOffSFQ + 4 * kTileScaleBytes;     // 4 x 512
 constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
 constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
 constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
-constexpr int kNumBars = 1 + 2 * kStages + 2 + 1 + 2 + 2;  // Q, K/V stage full+empty, S_full[2], S_free, P_full[2], O_done[2]
+constexpr int kNumBars = 4 + 2 * kStages + 2 + 1 + 2 + 2 + 2;  // Q full/empty[2], K/V stage full+empty, S_full[2], S_free, P_full[2], O_done[2], O_free[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
+#ifndef MXATTN_PERSIST_MAX_T
+#define MXATTN_PERSIST_MAX_T 16
+#endif
+constexpr int kPersistMaxTiles = MXATTN_PERSIST_MAX_T;    // longest key/value sequence (in tiles) run by the persistent variant
 constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
 
-enum Bar { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = BAR_KFULL + kStages,     // one full / empty pair per K/V stage
+enum Bar { BAR_Q = 0, BAR_QEMPTY = 2, BAR_KFULL = 4, BAR_KEMPTY = BAR_KFULL + kStages,     // one full / empty pair per K/V stage
            BAR_SFULL = BAR_KEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
-           BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2 };
+           BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2, BAR_OFREE = BAR_ODONE + 2 };
 
 // tensor-memory columns
 constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK = 424,
@@ -94,13 +98,19 @@ struct Params {
   uint8_t* dump;        // per-tile P-hat images, scales, running maxima and final row sums (debug entry point only)
   int64_t Nq, Nkv;
   int q_tiles, kv_tiles, q_pairs;
+  int total_items;      // B * H * q_pairs work items (one = two query tiles of one head)
   float scale_log2e;    // softmax_scale * log2(e)
   float softmax_scale;
 };
 
 // ---------------------------------------------------------------------------------------------
-template <bool kUos, bool kPnq, bool kOutF32, bool kDump>
+// kPersist: the CTA walks several work items (blockIdx.x, blockIdx.x + gridDim.x, ...) and keeps its barriers,
+// tensor memory and pipelines across them: the next item's Q tiles and first K/V tiles are fetched and its first
+// scores computed while the current item drains.  Used for short KV sequences, where the per-CTA set-up, the
+// latency of the first loads and the launch gap between CTAs are a large share of an item's time.
+template <bool kUos, bool kPnq, bool kOutF32, bool kDump, bool kPersist>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) {
+  static_assert(!(kDump && kPersist), "the tile dump is written by the one-item-per-CTA variant only");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -111,13 +121,14 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (*reinterpret_cast<volatile int*>(p.status) != 0) return;   // an earlier CTA gave up: drain the grid quickly
-  const int bh = blockIdx.x / p.q_pairs;
-  const int pair = blockIdx.x - bh * p.q_pairs;
   const int T = p.kv_tiles;
+  const int bh0 = blockIdx.x / p.q_pairs, pair0 = blockIdx.x - bh0 * p.q_pairs;
 
   // ---- setup -------------------------------------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar(BAR_Q), 1);
+    mbar_init(bar(BAR_Q + 0), 1); mbar_init(bar(BAR_Q + 1), 1);
+    mbar_init(bar(BAR_QEMPTY + 0), 1); mbar_init(bar(BAR_QEMPTY + 1), 1);
+    mbar_init(bar(BAR_OFREE + 0), 4 * kSplit); mbar_init(bar(BAR_OFREE + 1), 4 * kSplit);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(BAR_KFULL + s), 1); mbar_init(bar(BAR_KEMPTY + s), 1);
     }
@@ -150,40 +161,48 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   if (warp == kSoftmaxWarps) {
     // =============================== producer ===============================================
     if (lane == 0) {
-      const int64_t qt0 = (int64_t)bh * p.q_tiles + 2 * pair;
-      const int64_t qt1 = (2 * pair + 1 < p.q_tiles) ? qt0 + 1 : qt0;     // odd tail: reuse tile 0 (result unused)
-      mbar_expect_tx(bar(BAR_Q), 2 * (kTileCodeBytes + kTileScaleBytes));
-      bulk_g2s(sbase + kOffQ, p.q_codes + qt0 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q));
-      bulk_g2s(sbase + kOffQ + kTileCodeBytes, p.q_codes + qt1 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q));
-      bulk_g2s(sbase + kOffSFQ, p.q_scales + qt0 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q));
-      bulk_g2s(sbase + kOffSFQ + kTileScaleBytes, p.q_scales + qt1 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q));
-      const int64_t kv0 = (int64_t)bh * T;
-      int issued = 0;
+      int F = 0;                                   // tiles issued so far, over all items of this CTA
+      int q_issued = 0;                            // items whose Q tiles were issued
       bool ok = true;
-      for (int j = 0; j < T && ok; ++j) {
-        const int s = j % kStages;
-        const uint32_t ph = (uint32_t)((j / kStages) & 1);
-        if (j >= kStages) ok = mbar_wait(bar(BAR_KEMPTY + s), ph ^ 1u, abort_flag, p.status, 11);
+      for (int n = 0, item = blockIdx.x; (kPersist ? item < p.total_items : n < 1) && ok; ++n, item += gridDim.x) {
+        const int bh = item / p.q_pairs, pair = item - bh * p.q_pairs;
+        const int qb = kPersist ? (n & 1) : 0;     // Q buffer
+        // the Q buffer of item n - 2 is free once every GEMM 1 of that item has completed
+        if (kPersist && n >= 2) ok = mbar_wait(bar(BAR_QEMPTY + qb), (uint32_t)(((n - 2) >> 1) & 1), abort_flag, p.status, 13);
         if (!ok) break;
-        // K-hat_j and V-hat_j travel together: one full / one empty barrier per stage (the issuer thread's time
-        // per tile is what bounds the kernel, and every wait or commit it does not need shortens it)
-        mbar_expect_tx(bar(BAR_KFULL + s), 2 * (kTileCodeBytes + kTileScaleBytes));
-        bulk_g2s(sbase + kOffK + s * kTileCodeBytes, p.k_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
-        bulk_g2s(sbase + kOffSFK + s * kTileScaleBytes, p.k_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
-        bulk_g2s(sbase + kOffV + s * kVStageBytes, p.v_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
-        bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
-        issued = j + 1;
+        const int64_t qt0 = (int64_t)bh * p.q_tiles + 2 * pair;
+        const int64_t qt1 = (2 * pair + 1 < p.q_tiles) ? qt0 + 1 : qt0;     // odd tail: reuse tile 0 (result unused)
+        const uint32_t sq = sbase + kOffQ + qb * 2 * kTileCodeBytes, ssf = sbase + kOffSFQ + qb * 2 * kTileScaleBytes;
+        mbar_expect_tx(bar(BAR_Q + qb), 2 * (kTileCodeBytes + kTileScaleBytes));
+        bulk_g2s(sq, p.q_codes + qt0 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q + qb));
+        bulk_g2s(sq + kTileCodeBytes, p.q_codes + qt1 * kTileCodeBytes, kTileCodeBytes, bar(BAR_Q + qb));
+        bulk_g2s(ssf, p.q_scales + qt0 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q + qb));
+        bulk_g2s(ssf + kTileScaleBytes, p.q_scales + qt1 * kTileScaleBytes, kTileScaleBytes, bar(BAR_Q + qb));
+        q_issued = n + 1;
+        const int64_t kv0 = (int64_t)bh * T;
+        for (int j = 0; j < T && ok; ++j, ++F) {
+          const int s = F % kStages;
+          const uint32_t ph = (uint32_t)((F / kStages) & 1);
+          if (F >= kStages) ok = mbar_wait(bar(BAR_KEMPTY + s), ph ^ 1u, abort_flag, p.status, 11);
+          if (!ok) break;
+          // K-hat_j and V-hat_j travel together: one full / one empty barrier per stage (the issuer thread's time
+          // per tile is what bounds the kernel, and every wait or commit it does not need shortens it)
+          mbar_expect_tx(bar(BAR_KFULL + s), 2 * (kTileCodeBytes + kTileScaleBytes));
+          bulk_g2s(sbase + kOffK + s * kTileCodeBytes, p.k_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
+          bulk_g2s(sbase + kOffSFK + s * kTileScaleBytes, p.k_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
+          bulk_g2s(sbase + kOffV + s * kVStageBytes, p.v_codes + (kv0 + j) * kTileCodeBytes, kTileCodeBytes, bar(BAR_KFULL + s));
+          bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
+        }
       }
       if (!ok || *abort_flag) {
         // gave up: let copies already in flight land before the CTA's shared memory is released
-        for (int j = (issued > kStages ? issued - kStages : 0); j < issued; ++j) {
-          const int s = j % kStages;
-          const uint32_t ph = (uint32_t)((j / kStages) & 1);
-          const long long t0 = clock64();
-          while (!mbar_try(bar(BAR_KFULL + s), ph) && clock64() - t0 < 200000000LL) {}
-        }
         const long long t0 = clock64();
-        while (!mbar_try(bar(BAR_Q), 0) && clock64() - t0 < 200000000LL) {}
+        for (int f = (F > kStages ? F - kStages : 0); f < F; ++f)
+          while (!mbar_try(bar(BAR_KFULL + f % kStages), (uint32_t)((f / kStages) & 1)) && clock64() - t0 < 200000000LL) {}
+        for (int n = (q_issued > 2 ? q_issued - 2 : 0); n < q_issued; ++n) {
+          const int qb = kPersist ? (n & 1) : 0;
+          while (!mbar_try(bar(BAR_Q + qb), (uint32_t)((kPersist ? (n >> 1) : 0) & 1)) && clock64() - t0 < 200000000LL) {}
+        }
       }
     }
   } else if (warp == kSoftmaxWarps + 1) {
@@ -198,37 +217,56 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       const uint32_t q_lo = (sbase + kOffQ) >> 4, k_lo = (sbase + kOffK) >> 4;
       const uint32_t v_lo = (sbase + kOffV) >> 4, p_lo = (sbase + kOffP) >> 4;
       auto desc = [](uint32_t lo) { return ((uint64_t)kDescHiTile << 32) | lo; };
-      auto gemm1 = [&](int t, int j) {      // S = Q_t K_j^T
-        const uint32_t a = q_lo + (uint32_t)t * (kTileCodeBytes >> 4);
-        const uint32_t b = k_lo + (uint32_t)(j % kStages) * (kTileCodeBytes >> 4);
-        const uint32_t sfa = tmem + kColSFQ + 4 * t, sfb = tmem + kColSFK + 4 * (j & 1);
+      // A tile is named by its item n (0, 1, ... of this CTA), its index j inside the item and its index f among
+      // all tiles of the CTA (f = n T + j; f = j without kPersist).  Stages, slots and barrier parities follow f.
+      auto gemm1 = [&](int t, int n, int j, int f) {      // S = Q_t K_j^T
+        const int qb = kPersist ? (n & 1) : 0;
+        if (kPersist && t == 0 && j == 0 && n > 0) {
+          // first GEMM 1 of a new item: its Q tiles must have landed; every GEMM 1 of the previous item has been
+          // issued before this point, so the scale-factor columns of Q can be overwritten
+          if (!mbar_wait(bar(BAR_Q + qb), (uint32_t)((n >> 1) & 1), abort_flag, p.status, 21)) return false;
+          tc_fence_after();
+          tc_cp_sf(tmem + kColSFQ + 0, sbase + kOffSFQ + qb * 2 * kTileScaleBytes);
+          tc_cp_sf(tmem + kColSFQ + 4, sbase + kOffSFQ + (qb * 2 + 1) * kTileScaleBytes);
+        }
+        const uint32_t a = q_lo + (uint32_t)(qb * 2 + t) * (kTileCodeBytes >> 4);
+        const uint32_t b = k_lo + (uint32_t)(f % kStages) * (kTileCodeBytes >> 4);
+        const uint32_t sfa = tmem + kColSFQ + 4 * t, sfb = tmem + kColSFK + 4 * (f & 1);
         tc_mma(tmem + kColS, desc(a), desc(b), make_idesc(128, 0), sfa, sfb, 0u);
         tc_mma(tmem + kColS, desc(a + 2), desc(b + 2), make_idesc(128, 1), sfa, sfb, 1u);   // K 64..127: +32 bytes
         tc_commit(bar(BAR_SFULL + t));
+        if (kPersist && t == 1 && j == T - 1) tc_commit(bar(BAR_QEMPTY + qb));   // last reader of this item's Q tiles
+        return true;
       };
-      auto gemm2 = [&](int t, int j) {      // O_t += P_t [V_j | 1]
+      auto gemm2 = [&](int t, int n, int j, int f) {      // O_t += P_t [V_j | 1]
+        if (kPersist && j == 0 && n > 0) {
+          // the accumulator is about to be overwritten: the previous item's epilogue must have copied it out
+          if (!mbar_wait(bar(BAR_OFREE + t), (uint32_t)((n - 1) & 1), abort_flag, p.status, 27)) return false;
+          tc_fence_after();
+        }
         tc_cp_sf(tmem + kColSFP + 4 * t, sbase + kOffSFP + t * kTileScaleBytes);
         const uint32_t a = p_lo + (uint32_t)t * (kTileCodeBytes >> 4);
-        const uint32_t b = v_lo + (uint32_t)(j % kStages) * (kVStageBytes >> 4);
+        const uint32_t b = v_lo + (uint32_t)(f % kStages) * (kVStageBytes >> 4);
         const uint32_t d = tmem + (t ? kColO1 : kColO0);
-        const uint32_t sfa = tmem + kColSFP + 4 * t, sfb = tmem + kColSFV + 8 * (j & 1);
+        const uint32_t sfa = tmem + kColSFP + 4 * t, sfb = tmem + kColSFV + 8 * (f & 1);
         tc_mma(d, desc(a), desc(b), make_idesc(kNV, 0), sfa, sfb, j > 0 ? 1u : 0u);
         tc_mma(d, desc(a + 2), desc(b + 2), make_idesc(kNV, 1), sfa, sfb, 1u);
         tc_commit(bar(BAR_ODONE + t));
+        return true;
       };
-      // K-hat_j and V-hat_j have landed (and, unless `first`, the score buffer is free): one fence, then the scale
-      // atoms of both go to tensor memory -- V's two tiles ahead of its GEMM, which keeps that copy out of the
-      // path from "P is ready" to "GEMM 2 issued" (slot j & 1 was last read by the GEMMs of tile j - 2, issued before)
-      auto wait_kv = [&](int j, bool first) {
-        const int s = j % kStages;
-        if (!mbar_wait(bar(BAR_KFULL + s), (uint32_t)((j / kStages) & 1), abort_flag, p.status, 22)) return false;
+      // K-hat and V-hat of tile f have landed (and, unless `first`, the score buffer is free): one fence, then the
+      // scale atoms of both go to tensor memory -- V's two tiles ahead of its GEMM, which keeps that copy out of the
+      // path from "P is ready" to "GEMM 2 issued" (slot f & 1 was last read by the GEMMs of tile f - 2, issued before)
+      auto wait_kv = [&](int f, bool first) {
+        const int s = f % kStages;
+        if (!mbar_wait(bar(BAR_KFULL + s), (uint32_t)((f / kStages) & 1), abort_flag, p.status, 22)) return false;
         if (!first) {
           if (!mbar_wait(bar(BAR_SFREE), sfree_n & 1u, abort_flag, p.status, 23)) return false;
           ++sfree_n;
         }
         tc_fence_after();
-        tc_cp_sf(tmem + kColSFK + 4 * (j & 1), sbase + kOffSFK + s * kTileScaleBytes);
-        tc_cp_sf(tmem + kColSFV + 8 * (j & 1), sbase + kOffSFV + s * kTileScaleBytes);
+        tc_cp_sf(tmem + kColSFK + 4 * (f & 1), sbase + kOffSFK + s * kTileScaleBytes);
+        tc_cp_sf(tmem + kColSFV + 8 * (f & 1), sbase + kOffSFV + s * kTileScaleBytes);
         return true;
       };
       auto wait_sfree = [&]() {
@@ -244,38 +282,85 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         tc_cp_sf(tmem + kColSFV + 4, sbase + kOffSFOnes);        // scales of the ones rows, both slots
         tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
       }
-      // prologue: S(0,0), S(1,0), S(0,1)
-      ok = ok && wait_kv(0, true);
-      if (ok) gemm1(0, 0);
-      ok = ok && wait_sfree();
-      if (ok) gemm1(1, 0);
-      if (T > 1) {
-        ok = ok && wait_kv(1, false);
-        if (ok) gemm1(0, 1);
-      }
-      // unrolled by the number of stages: stage indices, parities and descriptor offsets become constants, and the
-      // thread's scalar instructions between its tcgen05 instructions are part of the kernel's critical path
-#pragma unroll 4
-      for (int j = 0; j < T && ok; ++j) {
-        const int s = j % kStages;
-        ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);     // V_j arrived with K_j
-        if (!ok) break;
-        tc_fence_after();
-        gemm2(0, j);
-        if (j + 1 < T) {
-          ok = wait_sfree();
-          if (!ok) break;
-          gemm1(1, j + 1);
+      if (!kPersist) {
+        // prologue: S(0,0), S(1,0), S(0,1)
+        ok = ok && wait_kv(0, true);
+        if (ok) gemm1(0, 0, 0, 0);
+        ok = ok && wait_sfree();
+        if (ok) gemm1(1, 0, 0, 0);
+        if (T > 1) {
+          ok = ok && wait_kv(1, false);
+          if (ok) gemm1(0, 0, 1, 1);
         }
-        ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
-        if (!ok) break;
-        tc_fence_after();
-        gemm2(1, j);
-        tc_commit(bar(BAR_KEMPTY + s));            // the last reader of stage s: K_j and V_j may be overwritten
-        if (j + 2 < T) {
-          ok = wait_kv(j + 2, false);
+        // unrolled by the number of stages: stage indices, parities and descriptor offsets become constants, and the
+        // thread's scalar instructions between its tcgen05 instructions are part of the kernel's critical path
+#pragma unroll 4
+        for (int j = 0; j < T && ok; ++j) {
+          const int s = j % kStages;
+          ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(j & 1), abort_flag, p.status, 24);     // V_j arrived with K_j
           if (!ok) break;
-          gemm1(0, j + 2);
+          tc_fence_after();
+          gemm2(0, 0, j, j);
+          if (j + 1 < T) {
+            ok = wait_sfree();
+            if (!ok) break;
+            gemm1(1, 0, j + 1, j + 1);
+          }
+          ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
+          if (!ok) break;
+          tc_fence_after();
+          gemm2(1, 0, j, j);
+          tc_commit(bar(BAR_KEMPTY + s));            // the last reader of stage s: K_j and V_j may be overwritten
+          if (j + 2 < T) {
+            ok = wait_kv(j + 2, false);
+            if (!ok) break;
+            gemm1(0, 0, j + 2, j + 2);
+          }
+        }
+      } else {
+        // The same instruction stream over all tiles of all items of this CTA, f = 0 .. F_end - 1: the scores of
+        // the next item's first tiles are issued while the current item's last tiles are still in the softmax warps.
+        const int n_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+        const int F_end = n_items * T;
+        int n0 = 0, j0 = 0;                          // tile f
+        int n1 = (T > 1) ? 0 : 1, j1 = (T > 1) ? 1 : 0;        // tile f + 1
+        int n2 = n1, j2 = j1 + 1;                    // tile f + 2
+        if (j2 == T) { j2 = 0; ++n2; }
+        ok = ok && wait_kv(0, true);
+        if (ok) ok = gemm1(0, 0, 0, 0);
+        ok = ok && wait_sfree();
+        if (ok) ok = gemm1(1, 0, 0, 0);
+        if (F_end > 1) {
+          ok = ok && wait_kv(1, false);
+          if (ok) ok = gemm1(0, n1, j1, 1);
+        }
+#pragma unroll 4
+        for (int f = 0; f < F_end && ok; ++f) {
+          ok = mbar_wait(bar(BAR_PFULL + 0), (uint32_t)(f & 1), abort_flag, p.status, 24);
+          if (!ok) break;
+          tc_fence_after();
+          ok = gemm2(0, n0, j0, f);
+          if (!ok) break;
+          if (f + 1 < F_end) {
+            ok = wait_sfree();
+            if (!ok) break;
+            ok = gemm1(1, n1, j1, f + 1);
+            if (!ok) break;
+          }
+          ok = mbar_wait(bar(BAR_PFULL + 1), (uint32_t)(f & 1), abort_flag, p.status, 26);
+          if (!ok) break;
+          tc_fence_after();
+          ok = gemm2(1, n0, j0, f);
+          if (!ok) break;
+          tc_commit(bar(BAR_KEMPTY + f % kStages));
+          if (f + 2 < F_end) {
+            ok = wait_kv(f + 2, false);
+            if (!ok) break;
+            ok = gemm1(0, n2, j2, f + 2);
+            if (!ok) break;
+          }
+          n0 = n1; j0 = j1; n1 = n2; j1 = j2;
+          if (++j2 == T) { j2 = 0; ++n2; }
         }
       }
     }
@@ -288,8 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     const uint32_t t_s = tmem + kColS + lane_addr + kCols * h;
     const uint32_t t_o = tmem + (t ? kColO1 : kColO0) + lane_addr;     // column 0 of this row's accumulator
     const float c = p.scale_log2e;
-    float m_run = -INFINITY;
-    float l_run = 0.0f;                            // direct placement only (this thread's 64 columns)
+    float m_run, l_run;                            // l_run: direct placement only (this thread's 64 columns)
     // shared-space byte addresses of this thread's slots: its two 16-byte code chunks, its two scale
     // bytes, and the half-row maximum exchange (own slot / partner's slot; + 2048 on odd tiles)
     const uint32_t aP0 = sbase + kOffP + t * kTileCodeBytes + tile_code_offset(row, 2 * h);
@@ -305,9 +389,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     // the pair barrier alone).  Their waits watch a flag that nothing sets, and raise the CTA's flag on expiry.
     volatile int* const own_limit_only = abort_flag + 1;
     bool ok = true;
+    // Work items of this CTA (exactly one without kPersist).  F0 = tiles of the earlier items: the parities of the
+    // barriers that complete once per tile follow F0 + j.  X0 counts the earlier exchanges through the half-row
+    // slots (one per tile, plus the row-sum exchange of direct placement), which alternate between two buffers.
+    int item = blockIdx.x, F0 = 0, X0 = 0;
+    do {
+    int bh = bh0, pair = pair0;                     // with kPersist: set in the epilogue, the only place that needs them
+    m_run = -INFINITY;
+    l_run = 0.0f;
 
     for (int j = 0; j < T; ++j) {
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)((F0 + j) & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[kCols];
@@ -341,20 +433,20 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
 #pragma unroll
       for (int b = 1; b < kBlocksPerThread; ++b) own_max = fmaxf(own_max, bmax[b]);
       // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
-      const uint32_t par = (uint32_t)(j & 1) * 2048u;
+      const uint32_t par = (uint32_t)((X0 + j) & 1) * 2048u;
       sts32f(aMaxOwn + par, own_max);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
       const float partner_max = lds32f(aMaxPartner + par);
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t or rescales
       // O_t; the probe of that barrier is issued while the partner's maximum is on its way
-      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1));
+      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1));
       const float m_new = max3(m_run, own_max, partner_max);   // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
         if (!ok) break;
       }
       tc_fence_after();
@@ -451,16 +543,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
     }
 
     // ---- epilogue: O = O~ / l (line 18) ----
-    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     float l = l_run;
     if (!kPnq) {                                   // add the partner's half of the row sum
-      const uint32_t par = (uint32_t)(T & 1) * 2048u;
+      const uint32_t par = (uint32_t)((X0 + T) & 1) * 2048u;
       sts32f(aMaxOwn + par, l_run);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       l = l_run + lds32f(aMaxPartner + par);
     }
     if (ok) {
       tc_fence_after();
+      if (kPersist) { bh = item / p.q_pairs; pair = item - bh * p.q_pairs; }
       const int qtile = 2 * pair + t;
       const int64_t grow = (int64_t)qtile * kTile + row;
       if (kPnq) {
@@ -472,7 +565,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
       const bool store = (qtile < p.q_tiles) && (grow < p.Nq);
       const float inv_l = 1.0f / l;                // line 18 as one reciprocal and 64 multiplies per thread
       if (kDump && h == 0 && qtile < p.q_tiles)
-        reinterpret_cast<float*>(p.dump + (int64_t)gridDim.x / p.q_pairs * p.q_tiles * T * kDumpTileBytes)
+        reinterpret_cast<float*>(p.dump + (int64_t)p.total_items / p.q_pairs * p.q_tiles * T * kDumpTileBytes)
             [((int64_t)bh * p.q_tiles + qtile) * kTile + row] = l;
       const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + kCols * h;
 #pragma unroll 1
@@ -502,7 +595,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
           }
         }
       }
+      if (kPersist) {                              // this row's accumulator has been read: GEMM 2 of the next item may overwrite it
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_OFREE + t));
+      }
     }
+    F0 += T;
+    X0 += T + (kPnq ? 0 : 1);
+    } while (kPersist && ok && (item += (int)gridDim.x) < p.total_items);
   }
 
   // ---- teardown ------------------------------------------------------------------------------
@@ -554,25 +655,38 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
   const int64_t pairs = (qt + 1) / 2;
   const int64_t grid = (int64_t)B * H * pairs;
   if (qt > 0x3FFFFFFF || kt > 0x3FFFFFFF || grid > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
-  p.q_tiles = (int)qt; p.kv_tiles = (int)kt; p.q_pairs = (int)pairs;
+  p.q_tiles = (int)qt; p.kv_tiles = (int)kt; p.q_pairs = (int)pairs; p.total_items = (int)grid;
   p.scale_log2e = softmax_scale * 1.4426950408889634f;
   p.softmax_scale = softmax_scale;
 
   const bool uos = flags & MXATTN_FLAG_UOS, pnq = flags & MXATTN_FLAG_PNQ, f32 = flags & MXATTN_FLAG_OUT_FP32;
+  // Short key/value sequences with more work items than SMs: one CTA per SM walks the items, so that the set-up,
+  // the first loads and the epilogue of one item overlap the tiles of its neighbours.  Long sequences keep one
+  // item per CTA (the hardware's block scheduler then balances the tail better than a static assignment).
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+      return MXATTN_ECUDA;
+    n_sm = v;
+  }
+  const bool persist = !dump && grid > n_sm && kt <= kPersistMaxTiles;
   void (*kern)(const Params) = nullptr;
-#define PICK(U, P, F) if (uos == U && pnq == P && f32 == F) kern = attention_kernel<U, P, F, false>;
+#define PICK(U, P, F)                                                                     \
+  if (uos == U && pnq == P && f32 == F)                                                   \
+    kern = persist ? attention_kernel<U, P, F, false, true> : attention_kernel<U, P, F, false, false>;
   PICK(false, false, false) PICK(false, false, true) PICK(false, true, false) PICK(false, true, true)
   PICK(true, false, false) PICK(true, false, true) PICK(true, true, false) PICK(true, true, true)
 #undef PICK
   if (dump) {                                     // debug entry point: fp32 output only
     if (!f32) return MXATTN_EINVAL;
-#define PICKD(U, P) if (uos == U && pnq == P) kern = attention_kernel<U, P, true, true>;
+#define PICKD(U, P) if (uos == U && pnq == P) kern = attention_kernel<U, P, true, true, false>;
     PICKD(false, false) PICKD(false, true) PICKD(true, false) PICKD(true, true)
 #undef PICKD
   }
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return MXATTN_ECUDA;
-  kern<<<(unsigned)grid, kThreads, kSmemBytes, stream>>>(p);
+  kern<<<(unsigned)(persist ? n_sm : grid), kThreads, kSmemBytes, stream>>>(p);
   count_launch(1);
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
 }

@@ -56,6 +56,30 @@ def test_ragged_shapes(nq, nkv):
     check(run_forward(cfg, q, k, v, True, True), oracle_out(cfg, q, k, v, True, True))
 
 
+# More work items (head x pair of query tiles) than the device has SMs and a short key/value sequence: the launch
+# uses the variant of the kernel in which one CTA per SM walks several items.  600 items give every CTA four or five
+# of them, so the double-buffered Q tiles and every barrier parity wrap at least once.
+@pytest.mark.parametrize("nkv,uos,pnq", [(100, True, True), (300, True, True), (300, False, False), (896, True, True),
+                                         (2500, True, False)])
+def test_many_short_items_per_cta(nkv, uos, pnq):
+    cfg = si.custom_config("p", 4, 30, 1100, nkv, 77 + nkv)
+    q, k, v = si.make_all(cfg)
+    check(run_forward(cfg, q, k, v, uos, pnq), oracle_out(cfg, q, k, v, uos, pnq))
+
+
+@pytest.mark.parametrize("uos,pnq", [(True, True), (True, False)])
+def test_item_walking_variant_is_bit_identical_to_one_item_per_cta(uos, pnq):
+    """The same head replicated 640 times (walked, several items per CTA) against a single copy of it (5 items on 5
+    CTAs): the arithmetic of a work item does not depend on which variant ran it."""
+    one = si.custom_config("p1", 1, 1, 1100, 700, 5)
+    q, k, v = si.make_all(one)
+    want = run_forward(one, q, k, v, uos, pnq)
+    many = si.custom_config("pm", 8, 80, 1100, 700, 5)
+    rep = lambda x: np.ascontiguousarray(np.broadcast_to(x, (many.B, many.H) + x.shape[2:]))
+    got = run_forward(many, rep(q), rep(k), rep(v), uos, pnq)
+    assert torch.equal(got, want.expand_as(got))
+
+
 @pytest.mark.parametrize("recipe", ["outlier", "wan", "hunyuan"])
 def test_structured_inputs_small(recipe):
     cfg = si.custom_config("s", 2, 2, 384, 1536, 41, recipe)
