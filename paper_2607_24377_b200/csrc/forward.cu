@@ -43,6 +43,11 @@
 // O_0 [128,272), O_1 [272,416), scale factors from 416.
 //
 // Every mbarrier wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
+#include <cuda.h>              // CUtensorMap and the enumerations of its encoder (types only: nothing links libcuda)
+#include <cudaTypedefs.h>
+
+#include <string.h>
+
 #include <type_traits>
 
 #include "common.cuh"
@@ -76,10 +81,14 @@ constexpr int kNumBars = 4 + 2 * kStages + 2 + 1 + 2 + 2 + 2;  // Q full/empty[2
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
 #ifndef MXATTN_PERSIST_MAX_T
-#define MXATTN_PERSIST_MAX_T 16
+#define MXATTN_PERSIST_MAX_T 20
 #endif
 constexpr int kPersistMaxTiles = MXATTN_PERSIST_MAX_T;    // longest key/value sequence (in tiles) run by the persistent variant
-constexpr int kSmemBytes = kOffMax + 2 * 2 * 2 * 128 * 4 + 1024;   // + slack for the 1024 alignment
+constexpr int kOffOut = (kOffMax + 2 * 2 * 2 * 128 * 4 + 1023) & ~1023;   // bf16 output staging: one box per softmax warp
+constexpr int kOutBoxBytes = 32 * kCols * 2;               // 32 rows x 64 bf16 (128 bytes, the span of the 128-byte swizzle)
+constexpr int kSmemBytes = kOffOut + kSoftmaxWarps * kOutBoxBytes + 1024;   // + slack for the 1024 alignment
+static_assert(kOffOut % 1024 == 0 && kOutBoxBytes % 1024 == 0, "swizzled boxes start on the swizzle pattern's period");
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 enum Bar { BAR_Q = 0, BAR_QEMPTY = 2, BAR_KFULL = 4, BAR_KEMPTY = BAR_KFULL + kStages,     // one full / empty pair per K/V stage
            BAR_SFULL = BAR_KEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
@@ -109,7 +118,7 @@ struct Params {
 // scores computed while the current item drains.  Used for short KV sequences, where the per-CTA set-up, the
 // latency of the first loads and the launch gap between CTAs are a large share of an item's time.
 template <bool kUos, bool kPnq, bool kOutF32, bool kDump, bool kPersist>
-__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, const __grid_constant__ CUtensorMap out_map) {
   static_assert(!(kDump && kPersist), "the tile dump is written by the one-item-per-CTA variant only");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -341,7 +350,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
           tc_fence_after();
           ok = gemm2(0, n0, j0, f);
           if (!ok) break;
-          if (f + 1 < F_end) {
+          // On the last tile of an item the score buffer is released only after the first group's epilogue, so
+          // the second group's GEMM 2 (and with it that group's epilogue) goes first there.
+          const bool item_end = (j0 == T - 1);
+          if (!item_end && f + 1 < F_end) {
             ok = wait_sfree();
             if (!ok) break;
             ok = gemm1(1, n1, j1, f + 1);
@@ -353,6 +365,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
           ok = gemm2(1, n0, j0, f);
           if (!ok) break;
           tc_commit(bar(BAR_KEMPTY + f % kStages));
+          if (item_end && f + 1 < F_end) {
+            ok = wait_sfree();
+            if (!ok) break;
+            ok = gemm1(1, n1, j1, f + 1);
+            if (!ok) break;
+          }
           if (f + 2 < F_end) {
             ok = wait_kv(f + 2, false);
             if (!ok) break;
@@ -568,31 +586,55 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
         reinterpret_cast<float*>(p.dump + (int64_t)p.total_items / p.q_pairs * p.q_tiles * T * kDumpTileBytes)
             [((int64_t)bh * p.q_tiles + qtile) * kTile + row] = l;
       const int64_t obase = ((int64_t)bh * p.Nq + grow) * kHeadDim + kCols * h;
+      if (kOutF32) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < kCols; c0 += 32) {
-        uint32_t r32[32];
-        TMEM_LD32(t_o + kCols * h + c0, r32);
-        tmem_ld_wait();
-        if (store) {
-          if (kOutF32) {
+        for (int c0 = 0; c0 < kCols; c0 += 32) {
+          uint32_t r32[32];
+          TMEM_LD32(t_o + kCols * h + c0, r32);
+          tmem_ld_wait();
+          if (store) {
             float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + obase + c0);
 #pragma unroll
             for (int i = 0; i < 8; ++i)
               dst[i] = make_float4(__uint_as_float(r32[4 * i]) * inv_l, __uint_as_float(r32[4 * i + 1]) * inv_l,
                                    __uint_as_float(r32[4 * i + 2]) * inv_l, __uint_as_float(r32[4 * i + 3]) * inv_l);
-          } else {
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + obase + c0);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint32_t hh[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float a = __uint_as_float(r32[8 * i + 2 * k]) * inv_l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) * inv_l;
-                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hh[k]) : "f"(b2), "f"(a));
-              }
-              dst[i] = make_uint4(hh[0], hh[1], hh[2], hh[3]);
-            }
           }
+        }
+      } else {
+        // bf16: the warp's 32 half rows (128 bytes each) go to shared memory and from there to global memory as one
+        // tensor copy (box of 32 rows x 64 columns; rows at or beyond Nq are clipped by the copy).  Written from
+        // registers, a warp's 16-byte stores land 256 bytes apart (one partly filled sector per lane and
+        // instruction); and any store instruction of these warps queues 64 KiB per item in front of the next
+        // tile's shared-memory traffic.  The box uses the 128-byte swizzle (16-byte chunk c of row r sits at
+        // chunk c ^ (r & 7)), which also spreads a quarter warp's stores over all banks.
+        const uint32_t aBox = sbase + kOffOut + (t * 8 + h * 4 + (row >> 5)) * kOutBoxBytes;    // one box per warp
+        const uint32_t aRow = aBox + (row & 31) * (kCols * 2);
+        if (kPersist) {                              // the previous item's copy has read the box
+          if ((row & 31) == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
+        }
+#pragma unroll 1
+        for (int c0 = 0; c0 < kCols; c0 += 32) {
+          uint32_t r32[32];
+          TMEM_LD32(t_o + kCols * h + c0, r32);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint32_t hh[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float a = __uint_as_float(r32[8 * i + 2 * k]) * inv_l, b2 = __uint_as_float(r32[8 * i + 2 * k + 1]) * inv_l;
+              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hh[k]) : "f"(b2), "f"(a));
+            }
+            sts128(aRow + ((((c0 >> 3) + i) ^ (row & 7)) << 4), make_uint4(hh[0], hh[1], hh[2], hh[3]));
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if ((row & 31) == 0 && qtile < p.q_tiles && (int64_t)qtile * kTile + (row & ~31) < p.Nq) {
+          asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                       ::"l"(&out_map), "r"(kCols * h), "r"(qtile * kTile + (row & ~31)), "r"(bh), "r"(aBox) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
       if (kPersist) {                              // this row's accumulator has been read: GEMM 2 of the next item may overwrite it
@@ -607,6 +649,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p) 
   }
 
   // ---- teardown ------------------------------------------------------------------------------
+  if (!kOutF32 && warp < kSoftmaxWarps && lane == 0)
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // the output copies have left shared memory
   tc_fence_before();
   __syncthreads();
   if (warp == kSoftmaxWarps + 1) {
@@ -671,7 +715,29 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
     n_sm = v;
   }
   const bool persist = !dump && grid > n_sm && kt <= kPersistMaxTiles;
-  void (*kern)(const Params) = nullptr;
+  // Descriptor of the bf16 output as a [B H][Nq][128] tensor with boxes of 32 rows x 64 columns (the epilogue's copies).
+  CUtensorMap out_map;
+  memset(&out_map, 0, sizeof(out_map));
+  if (!f32) {
+    static PFN_cuTensorMapEncodeTiled encode = nullptr;
+    if (!encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || !fn)
+        return MXATTN_ECUDA;
+      encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+    }
+    if (Nq > 0x7FFFFFFFLL || (uint64_t)Nq * kHeadDim * 2 >= (1ULL << 40)) return MXATTN_EUNSUPPORTED;
+    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)Nq, (cuuint64_t)B * H};
+    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)Nq * kHeadDim * 2};     // bytes, dimensions 1 and 2
+    const cuuint32_t box[3] = {(cuuint32_t)kCols, 32u, 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    if (encode(&out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, o, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return MXATTN_ECUDA;
+  }
+  void (*kern)(const Params, const CUtensorMap) = nullptr;
 #define PICK(U, P, F)                                                                     \
   if (uos == U && pnq == P && f32 == F)                                                   \
     kern = persist ? attention_kernel<U, P, F, false, true> : attention_kernel<U, P, F, false, false>;
@@ -686,7 +752,7 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
   }
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return MXATTN_ECUDA;
-  kern<<<(unsigned)(persist ? n_sm : grid), kThreads, kSmemBytes, stream>>>(p);
+  kern<<<(unsigned)(persist ? n_sm : grid), kThreads, kSmemBytes, stream>>>(p, out_map);
   count_launch(1);
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
 }
