@@ -90,10 +90,8 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {     /
 // the CTA already gave up); the caller then skips to the teardown.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at full clock
 // `abort_flag` is the flag the wait watches; `raise_flag`, if given, is the one it sets on expiry instead.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code, long long limit = kWaitLimitCycles,
-                                          volatile int* raise_flag = nullptr) {
-  if (mbar_try(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_wait_loop(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int* status, int code, long long limit, volatile int* raise_flag) {
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
@@ -106,6 +104,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status, int code, long long limit = kWaitLimitCycles,
+                                          volatile int* raise_flag = nullptr) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_loop(bar, parity, abort_flag, status, code, limit, raise_flag);
+}
+// The same wait with its loop out of line, for the single-thread roles (copy producer, MMA issuer): their time per
+// tile grows with the amount of code they walk through, not only with the instructions they execute, and this keeps
+// one try_wait and a branch per wait in their loops.  (In the softmax warps, which run at the register limit, the
+// call's register conventions cost more than the compact code gains.)
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                   int* status, int code) {
+  return mbar_wait_loop(bar, parity, abort_flag, status, code, kWaitLimitCycles, nullptr);
+}
+__device__ __forceinline__ bool mbar_wait1(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
