@@ -32,9 +32,9 @@ NOMINAL_FP4_TFLOPS = 9000.0      # dense FP4, nominal
 FP4_OVER_BF16 = 4.0              # nominal ratio of dense FP4 to dense bf16 tensor throughput
 QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0
 # DRAM bytes of one attention launch, from the ncu capture of the same kernel on sweep16384
-# (253.0 MB, profiles/attention_kernel_sweep16384.txt) scaled by tokens x heads (traffic follows the
-# operand bytes, not the flops).
-ATTN_TRAFFIC_PER_TOKEN_HEAD = 253.0e6 / (16384 * 40)
+# (259.4 MB, profiles/attention_kernel_sweep16384.txt) scaled by tokens x heads (traffic follows the
+# operand bytes, not the flops; valid for the self-attention workloads, Nq = Nkv).
+ATTN_TRAFFIC_PER_TOKEN_HEAD = 259.4e6 / (16384 * 40)
 
 
 def load_peaks():
@@ -354,7 +354,7 @@ def main():
         "e2e": e2e, "gpu_launches": 4 * args.steps,
         "roofline": {"bound": "tensor", "kernel": "attention_kernel<uos,pnq>", "achieved": attn_tflops,
                      "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak,
-                     "traffic": ATTN_TRAFFIC_PER_TOKEN_HEAD * Nkv * B * H,
+                     "traffic": ATTN_TRAFFIC_PER_TOKEN_HEAD * Nkv * B * H if Nq == Nkv else None,
                      "traffic_note": "ncu dram bytes of a sweep16384 launch scaled by tokens x heads",
                      "peak_note": f"dense FP4 = {peaks['source']} sustained bf16 cuBLAS {peaks['bf16_tflops_sustained']} x nominal ratio 4 (of {peaks['source']})",
                      "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms,

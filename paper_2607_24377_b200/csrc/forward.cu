@@ -42,6 +42,14 @@
 // to registers at once, so the buffer is free again long before the other group needs it),
 // O_0 [128,272), O_1 [272,416), scale factors from 416.
 //
+// Epilogue: O = O~ / l; the bf16 result is staged in shared memory (one 32-row x 128-byte box per softmax warp,
+// 128-byte swizzle) and leaves as one tensor copy per warp through a tensor map of the output, so that whole
+// lines are written and the stores do not queue in front of the next tile's shared-memory traffic.
+//
+// Two launch shapes: one CTA per work item (two query tiles of one head), or -- more items than SMs and a short
+// KV sequence -- one CTA per SM that walks the items and keeps barriers, tensor memory and the K/V ring across
+// them (template flag kPersist).
+//
 // Every mbarrier wait is bounded; on expiry the CTA records a code in `status`, drains and exits.
 #include <cuda.h>              // CUtensorMap and the enumerations of its encoder (types only: nothing links libcuda)
 #include <cudaTypedefs.h>
