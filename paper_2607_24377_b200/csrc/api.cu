@@ -175,7 +175,7 @@ extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_sc
 // kernels of head h (PCIe is full duplex).  The two helper streams and the events are created on
 // first use, once per device, and kept for the life of the process; no device memory is allocated.
 struct HostPipe {
-  cudaStream_t in = nullptr, quant = nullptr, out = nullptr;
+  cudaStream_t in = nullptr, quant = nullptr, out = nullptr, attn = nullptr;
   std::vector<cudaEvent_t> ev;
 };
 static HostPipe g_pipe[64];
@@ -187,6 +187,7 @@ static HostPipe* host_pipe(size_t n_events) {
   if (!hp.in && cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   if (!hp.out && cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   if (!hp.quant && cudaStreamCreateWithFlags(&hp.quant, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (!hp.attn && cudaStreamCreateWithFlags(&hp.attn, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   while (hp.ev.size() < n_events) {
     cudaEvent_t e;
     if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
@@ -195,25 +196,26 @@ static HostPipe* host_pipe(size_t n_events) {
   return &hp;
 }
 
-// How many heads one pipeline stage of mxattn_forward_host takes.  A stage is one attention launch of
-// g * ceil(ceil(Nq/128)/2) CTAs on an n_sm-SM device: a partially filled last wave costs as much as a full
-// one (hunyuan: 466 CTAs per head = 3.15 waves on 148 SMs, 27 % lost at g = 1), while a larger g exposes more of
-// the first stage's host-to-device copy and of the last stage's device-to-host copy.  The estimate below
-// (attention at ~1.6 PFLOP/s, copies at ~50 GB/s) only has to rank the candidates.
-static int heads_per_stage(size_t bh, int64_t Nq, int64_t Nkv, size_t in_bytes_per_head, size_t out_bytes_per_head) {
+// How many heads a pipeline stage of mxattn_forward_host takes (after the first stage, which takes one).  A stage
+// is one attention launch of g * ceil(ceil(Nq/128)/2) CTAs.  Consecutive stages' launches go to two streams, so
+// the CTAs of the next stage start on the SMs the current one leaves and a partly filled last wave costs
+// nothing; what is left to weigh is a launch that cannot fill the device at all (small heads: take several),
+// the fixed cost per stage, and the last stage's copy out, which nothing hides.  The estimate (attention at
+// ~1.8 PFLOP/s, copies at ~50 GB/s, 20 us of launches and events per stage) only has to rank the candidates.
+static int heads_per_stage(size_t bh, int64_t Nq, int64_t Nkv, size_t out_bytes_per_head) {
   int dev = 0, n_sm = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (n_sm <= 0) n_sm = 148;
   const double ctas = (double)(((Nq + kTile - 1) / kTile + 1) / 2);
-  const double t_head = 4.0 * (double)Nq * (double)Nkv * kHeadDim / 1.6e15;
-  const double t_in = (double)in_bytes_per_head / 50e9, t_out = (double)out_bytes_per_head / 50e9;
+  const double t_head = 4.0 * (double)Nq * (double)Nkv * kHeadDim / 1.8e15;
+  const double t_out = (double)out_bytes_per_head / 50e9;
   int best = 1;
   double best_t = 1e300;
   for (int g = 1; g <= 8 && (size_t)g <= bh; ++g) {
     if (g > 1 && bh / g < 3) break;                 // keep at least three stages to overlap
-    const double waves = g * ctas / n_sm;
-    const double eff = waves / (double)(int64_t)(waves + 0.999999);
-    const double t = (double)bh * t_head / eff + g * (t_in + t_out);
+    const double fill = g * ctas / n_sm;
+    const double eff = fill < 1.0 ? fill : 1.0;
+    const double t = (double)bh * t_head / eff + g * t_out + 20e-6 * (double)((bh + g - 1) / g);
     if (t < best_t * 0.995) { best_t = t; best = g; }
   }
   return best;
@@ -248,8 +250,14 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   uint8_t* dv = dk + align_up(bh * kh, 256);
   uint8_t* dout = dv + align_up(bh * kh, 256);
   uint8_t* ws = dout + align_up(bh * oh, 256);
-  const int g = heads_per_stage(bh, Nq, Nkv, qh + 2 * kh, oh);
-  const size_t stages = (bh + g - 1) / g;
+  // The first stage takes one head (nothing hides its copy in), the others g heads each.
+  const int g = heads_per_stage(bh, Nq, Nkv, oh);
+  const size_t stages = (g == 1) ? bh : 1 + (bh - 1 + g - 1) / g;
+  auto first_head = [&](size_t st) {
+    if (g == 1 || st == 0) return st;
+    const size_t h = 1 + (st - 1) * (size_t)g;
+    return h < bh ? h : bh;
+  };
   HostPipe* hp = host_pipe(3 * stages + 2);
   if (!hp) return MXATTN_ECUDA;
   cudaEvent_t* ev = hp->ev.data();
@@ -257,10 +265,13 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   auto ck = [&](cudaError_t e) { if (e != cudaSuccess) fail = true; };
   ck(cudaEventRecord(ev[3 * stages], stream));                   // work already queued on the caller's stream comes first
   ck(cudaStreamWaitEvent(hp->in, ev[3 * stages], 0));
+  ck(cudaStreamWaitEvent(hp->attn, ev[3 * stages], 0));
   int rc = MXATTN_OK;
   for (size_t st = 0; st < stages && !fail && rc == MXATTN_OK; ++st) {
-    const size_t i = st * g;                                     // first head of the stage; heads are contiguous in memory
-    const size_t n = (bh - i < (size_t)g) ? bh - i : (size_t)g;
+    const size_t i = first_head(st), n = first_head(st + 1) - i;  // heads of the stage; heads are contiguous in memory
+    // attention launches alternate between the caller's stream and one of the pipeline's, so that the CTAs of a
+    // stage start on the SMs the previous stage's last CTAs leave (no tail, no launch gap between stages)
+    cudaStream_t as = (st & 1) ? hp->attn : stream;
     ck(cudaMemcpyAsync(dq + i * qh, static_cast<const char*>(q_host) + i * qh, n * qh, cudaMemcpyHostToDevice, hp->in));
     ck(cudaMemcpyAsync(dk + i * kh, static_cast<const char*>(k_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
     ck(cudaMemcpyAsync(dv + i * kh, static_cast<const char*>(v_host) + i * kh, n * kh, cudaMemcpyHostToDevice, hp->in));
@@ -270,8 +281,8 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
     // n heads); its operands are quantized on a stream of their own, behind the copies and ahead of the attention
     // launch, so that they fill the SMs the previous stage's attention kernel frees as it drains
     rc = forward_ws(dq + i * qh, dk + i * kh, dv + i * kh, dout + i * oh, 1, (int)n, Nq, Nkv, d, softmax_scale, flags,
-                    ws + i * w.total, n * w.total, stream, nullptr, hp->quant, ev[3 * st + 1]);
-    ck(cudaEventRecord(ev[3 * st + 2], stream));
+                    ws + i * w.total, n * w.total, as, nullptr, hp->quant, ev[3 * st + 1]);
+    ck(cudaEventRecord(ev[3 * st + 2], as));
     ck(cudaStreamWaitEvent(hp->out, ev[3 * st + 2], 0));
     ck(cudaMemcpyAsync(static_cast<char*>(o_host) + i * oh, dout + i * oh, n * oh, cudaMemcpyDeviceToHost, hp->out));
   }
@@ -281,13 +292,16 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   ck(cudaStreamSynchronize(hp->in));
   ck(cudaStreamSynchronize(hp->quant));
   ck(cudaStreamSynchronize(stream));
+  ck(cudaStreamSynchronize(hp->attn));
   ck(cudaStreamSynchronize(hp->out));
   g_launches = 4 * (int)stages;
   if (rc != MXATTN_OK) return rc;
   if (fail) return MXATTN_ECUDA;
   // one status word per stage, at the start of its workspace slice
   std::vector<int> stw(stages, 0);
-  if (cudaMemcpy2D(stw.data(), sizeof(int), ws, (size_t)g * w.total, sizeof(int), stages, cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaMemcpy(stw.data(), ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
+  if (stages > 1 && cudaMemcpy2D(stw.data() + 1, sizeof(int), ws + first_head(1) * w.total, (size_t)g * w.total, sizeof(int),
+                                 stages - 1, cudaMemcpyDeviceToHost) != cudaSuccess) return MXATTN_ECUDA;
   for (size_t i = 0; i < stages; ++i)
     if (stw[i]) return MXATTN_ETIMEOUT;
   return MXATTN_OK;
