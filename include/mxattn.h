@@ -203,11 +203,13 @@ int mxattn_forward_bf16(const void* q, const void* k, const void* v, void* o,
 size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags);
 
 /* End-to-end form for callers whose tensors live in HOST memory (pinned memory, so that the copies
- * are asynchronous): runs mxattn_forward_ws in stages of one or more heads (as many as it takes to fill
- * the GPU's SMs with whole waves of CTAs) out of `device_arena` and writes o into o_host.  The stages are
- * pipelined over the caller's `stream` (kernels) and two helper streams that the
- * library creates once per device (host->device copies of the next stage and the device->host copy of
- * the previous one overlap the kernels).  Work already queued on `stream` is waited for first;
+ * are asynchronous): runs mxattn_forward_ws in stages of one or more heads (one head first, then as many
+ * per stage as it takes to fill the GPU's SMs) out of `device_arena` and writes o into o_host.  The stages
+ * are pipelined over the caller's `stream` and four helper streams that the library creates once per
+ * device: host->device copies of the next stages, their quantization, and the device->host copy of the
+ * previous stage overlap the attention kernels, whose launches alternate between `stream` and a helper
+ * stream so that one stage's CTAs start as the previous stage's finish.  Work already queued on `stream`
+ * is waited for first;
  * the call returns after everything has finished (it SYNCHRONIZES).  `device_arena` is caller-owned
  * device memory of at least mxattn_forward_host_arena_bytes(); no device memory is allocated.
  * Returns MXATTN_ETIMEOUT if a bounded device-side wait expired in any head. */
