@@ -573,6 +573,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     }
 
     // ---- epilogue: O = O~ / l (line 18) ----
+    if (kPersist && !kOutF32) {                    // the previous item's output copy has read this warp's box
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+    }
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     float l = l_run;
     if (!kPnq) {                                   // add the partner's half of the row sum
@@ -586,6 +590,39 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       if (kPersist) { bh = item / p.q_pairs; pair = item - bh * p.q_pairs; }
       const int qtile = 2 * pair + t;
       const int64_t grow = (int64_t)qtile * kTile + row;
+      if (kPersist && !kOutF32) {
+        // Item-walking variant: the epilogue is part of every item's critical path.  Row sum and all 64 accumulator
+        // columns are loaded with one wait, the accumulator is handed back to the issuer at once, then the bf16
+        // rows go to this warp's swizzled box and out as one tensor copy (see the comments of the general path).
+        uint32_t lr = 0, r64[kCols];
+        if (kPnq) asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
+        TMEM_LD64(t_o + kCols * h, r64);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_OFREE + t));   // GEMM 2 of the next item may overwrite the accumulator
+        if (kPnq) l = __uint_as_float(lr);
+        const float inv_l = 1.0f / l;
+        const uint32_t aBox = sbase + kOffOut + (t * 8 + h * 4 + (row >> 5)) * kOutBoxBytes;
+        const uint32_t aRow = aBox + (row & 31) * (kCols * 2);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          uint32_t hh[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float a = __uint_as_float(r64[8 * i + 2 * k]) * inv_l, b2 = __uint_as_float(r64[8 * i + 2 * k + 1]) * inv_l;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hh[k]) : "f"(b2), "f"(a));
+          }
+          sts128(aRow + ((i ^ (row & 7)) << 4), make_uint4(hh[0], hh[1], hh[2], hh[3]));
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && qtile < p.q_tiles && (int64_t)qtile * kTile + (row & ~31) < p.Nq) {
+          asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                       ::"l"(&out_map), "r"(kCols * h), "r"(qtile * kTile + (row & ~31)), "r"(bh), "r"(aBox) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      } else {
       if (kPnq) {
         uint32_t lr;
         asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
@@ -621,10 +658,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
         // chunk c ^ (r & 7)), which also spreads a quarter warp's stores over all banks.
         const uint32_t aBox = sbase + kOffOut + (t * 8 + h * 4 + (row >> 5)) * kOutBoxBytes;    // one box per warp
         const uint32_t aRow = aBox + (row & 31) * (kCols * 2);
-        if (kPersist) {                              // the previous item's copy has read the box
-          if ((row & 31) == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          __syncwarp();
-        }
 #pragma unroll 1
         for (int c0 = 0; c0 < kCols; c0 += 32) {
           uint32_t r32[32];
@@ -653,6 +686,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(BAR_OFREE + t));
+      }
       }
     }
     F0 += T;
