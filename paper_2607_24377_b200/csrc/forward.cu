@@ -85,11 +85,11 @@ constexpr int kOffSFV = kOffSFK + kStages * kTileScaleBytes;   // 4 x 512
 constexpr int kOffSFOnes = kOffSFV + kStages * kTileScaleBytes; // 512
 constexpr int kOffSFP = kOffSFOnes + kTileScaleBytes;      // 2 x 512
 constexpr int kOffBar = kOffSFP + 2 * kTileScaleBytes;     // barriers
-constexpr int kNumBars = 4 + 2 * kStages + 2 + 1 + 2 + 2 + 2;  // Q full/empty[2], K/V stage full+empty, S_full[2], S_free, P_full[2], O_done[2], O_free[2]
+constexpr int kNumBars = 4 + 2 * kStages + 2 + 1 + 2 + 2;  // Q full/empty[2], K/V stage full+empty, S_full[2], S_free, P_full[2], O_done[2]
 constexpr int kOffMisc = kOffBar + kNumBars * 8;           // tmem slot, abort flag
 constexpr int kOffMax = kOffMisc + 64;                     // half-row maxima: [parity 2][tile 2][half 2][128] floats
 #ifndef MXATTN_PERSIST_MAX_T
-#define MXATTN_PERSIST_MAX_T 32
+#define MXATTN_PERSIST_MAX_T 48
 #endif
 constexpr int kPersistMaxTiles = MXATTN_PERSIST_MAX_T;    // longest key/value sequence (in tiles) run by the persistent variant
 constexpr int kOffOut = (kOffMax + 2 * 2 * 2 * 128 * 4 + 1023) & ~1023;   // bf16 output staging: one box per softmax warp
@@ -100,7 +100,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 enum Bar { BAR_Q = 0, BAR_QEMPTY = 2, BAR_KFULL = 4, BAR_KEMPTY = BAR_KFULL + kStages,     // one full / empty pair per K/V stage
            BAR_SFULL = BAR_KEMPTY + kStages, BAR_SFREE = BAR_SFULL + 2,
-           BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2, BAR_OFREE = BAR_ODONE + 2 };
+           BAR_PFULL = BAR_SFREE + 1, BAR_ODONE = BAR_PFULL + 2 };
 
 // tensor-memory columns
 constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK = 424,
@@ -149,7 +149,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
   if (tid == 0) {
     mbar_init(bar(BAR_Q + 0), 1); mbar_init(bar(BAR_Q + 1), 1);
     mbar_init(bar(BAR_QEMPTY + 0), 1); mbar_init(bar(BAR_QEMPTY + 1), 1);
-    mbar_init(bar(BAR_OFREE + 0), 4 * kSplit); mbar_init(bar(BAR_OFREE + 1), 4 * kSplit);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(BAR_KFULL + s), 1); mbar_init(bar(BAR_KEMPTY + s), 1);
     }
@@ -241,30 +240,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       // A tile is named by its item n (0, 1, ... of this CTA), its index j inside the item and its index f among
       // all tiles of the CTA (f = n T + j; f = j without kPersist).  Stages, slots and barrier parities follow f.
       auto gemm1 = [&](int t, int n, int j, int f) {      // S = Q_t K_j^T
-        const int qb = kPersist ? (n & 1) : 0;
-        if (kPersist && t == 0 && j == 0 && n > 0) {
-          // first GEMM 1 of a new item: its Q tiles must have landed; every GEMM 1 of the previous item has been
-          // issued before this point, so the scale-factor columns of Q can be overwritten
-          if (!MBAR_WAIT_ROLE(bar(BAR_Q + qb), (uint32_t)((n >> 1) & 1), abort_flag, p.status, 21)) return false;
-          tc_fence_after();
-          tc_cp_sf(tmem + kColSFQ + 0, sbase + kOffSFQ + qb * 2 * kTileScaleBytes);
-          tc_cp_sf(tmem + kColSFQ + 4, sbase + kOffSFQ + (qb * 2 + 1) * kTileScaleBytes);
-        }
-        const uint32_t a = q_lo + (uint32_t)(qb * 2 + t) * (kTileCodeBytes >> 4);
+        const uint32_t a = q_lo + (uint32_t)t * (kTileCodeBytes >> 4);
         const uint32_t b = k_lo + (uint32_t)(f % kStages) * (kTileCodeBytes >> 4);
         const uint32_t sfa = tmem + kColSFQ + 4 * t, sfb = tmem + kColSFK + 4 * (f & 1);
         tc_mma(tmem + kColS, desc(a), desc(b), make_idesc(128, 0), sfa, sfb, 0u);
         tc_mma(tmem + kColS, desc(a + 2), desc(b + 2), make_idesc(128, 1), sfa, sfb, 1u);   // K 64..127: +32 bytes
         tc_commit(bar(BAR_SFULL + t));
-        if (kPersist && t == 1 && j == T - 1) tc_commit(bar(BAR_QEMPTY + qb));   // last reader of this item's Q tiles
         return true;
       };
       auto gemm2 = [&](int t, int n, int j, int f) {      // O_t += P_t [V_j | 1]
-        if (kPersist && j == 0 && n > 0) {
-          // the accumulator is about to be overwritten: the previous item's epilogue must have copied it out
-          if (!MBAR_WAIT_ROLE(bar(BAR_OFREE + t), (uint32_t)((n - 1) & 1), abort_flag, p.status, 27)) return false;
-          tc_fence_after();
-        }
         tc_cp_sf(tmem + kColSFP + 4 * t, sbase + kOffSFP + t * kTileScaleBytes);
         const uint32_t a = p_lo + (uint32_t)t * (kTileCodeBytes >> 4);
         const uint32_t b = v_lo + (uint32_t)(f % kStages) * (kVStageBytes >> 4);
@@ -341,56 +325,76 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       } else {
         // The same instruction stream over all tiles of all items of this CTA, f = 0 .. F_end - 1: the scores of
         // the next item's first tiles are issued while the current item's last tiles are still in the softmax warps.
+        // Per tile the thread keeps one cursor (item n0, tile j0 of tile f) and derives two flags from it; what an
+        // item boundary adds is then one branch per GEMM 1.  `edge` of a GEMM 1 means: for query tile 0, the first
+        // tile of an item other than the CTA's first (wait for its Q tiles, copy their scales: every GEMM 1 of the
+        // previous item has been issued by then); for query tile 1, the last tile of its item (release the Q buffer).
+        // No barrier guards the accumulators across items: GEMM 2 of an item's first tile waits for that tile's
+        // P-hat, which the group's warps publish after their epilogue has read the previous item's accumulator.
         const int n_items = (p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
         const int F_end = n_items * T;
+        auto gemm1p = [&](int t, int n, int f, bool edge) {      // n: the item of tile f
+          const int qb = n & 1;
+          if (t == 0 && edge) {
+            if (!mbar_wait1(bar(BAR_Q + qb), (uint32_t)((n >> 1) & 1), abort_flag, p.status, 21)) return false;
+            tc_fence_after();
+            tc_cp_sf(tmem + kColSFQ + 0, sbase + kOffSFQ + qb * 2 * kTileScaleBytes);
+            tc_cp_sf(tmem + kColSFQ + 4, sbase + kOffSFQ + (qb * 2 + 1) * kTileScaleBytes);
+          }
+          const uint32_t a = q_lo + (uint32_t)(qb * 2 + t) * (kTileCodeBytes >> 4);
+          const uint32_t b = k_lo + (uint32_t)(f % kStages) * (kTileCodeBytes >> 4);
+          const uint32_t sfa = tmem + kColSFQ + 4 * t, sfb = tmem + kColSFK + 4 * (f & 1);
+          tc_mma(tmem + kColS, desc(a), desc(b), make_idesc(128, 0), sfa, sfb, 0u);
+          tc_mma(tmem + kColS, desc(a + 2), desc(b + 2), make_idesc(128, 1), sfa, sfb, 1u);
+          tc_commit(bar(BAR_SFULL + t));
+          if (t == 1 && edge) tc_commit(bar(BAR_QEMPTY + qb));
+          return true;
+        };
+        const bool one = (T == 1);
         int n0 = 0, j0 = 0;                          // tile f
-        int n1 = (T > 1) ? 0 : 1, j1 = (T > 1) ? 1 : 0;        // tile f + 1
-        int n2 = n1, j2 = j1 + 1;                    // tile f + 2
-        if (j2 == T) { j2 = 0; ++n2; }
         ok = ok && wait_kv(0, true);
-        if (ok) ok = gemm1(0, 0, 0, 0);
+        if (ok) ok = gemm1p(0, 0, 0, false);
         ok = ok && wait_sfree();
-        if (ok) ok = gemm1(1, 0, 0, 0);
+        if (ok) ok = gemm1p(1, 0, 0, one);
         if (F_end > 1) {
           ok = ok && wait_kv(1, false);
-          if (ok) ok = gemm1(0, n1, j1, 1);
+          if (ok) ok = gemm1p(0, one ? 1 : 0, 1, one);
         }
 #pragma unroll 4
         for (int f = 0; f < F_end && ok; ++f) {
-          ok = MBAR_WAIT_ROLE(bar(BAR_PFULL + 0), (uint32_t)(f & 1), abort_flag, p.status, 24);
+          const bool item_end = (j0 == T - 1);       // tile f + 1 starts an item
+          const bool pre_end = one || (j0 == T - 2); // tile f + 1 ends an item, tile f + 2 starts one
+          const int n1 = n0 + (item_end ? 1 : 0), n2 = n1 + (pre_end ? 1 : 0);
+          ok = mbar_wait1(bar(BAR_PFULL + 0), (uint32_t)(f & 1), abort_flag, p.status, 24);
           if (!ok) break;
           tc_fence_after();
-          ok = gemm2(0, n0, j0, f);
-          if (!ok) break;
+          gemm2(0, 0, j0, f);
           // On the last tile of an item the score buffer is released only after the first group's epilogue, so
           // the second group's GEMM 2 (and with it that group's epilogue) goes first there.
-          const bool item_end = (j0 == T - 1);
           if (!item_end && f + 1 < F_end) {
             ok = wait_sfree();
             if (!ok) break;
-            ok = gemm1(1, n1, j1, f + 1);
+            ok = gemm1p(1, n1, f + 1, pre_end);
             if (!ok) break;
           }
-          ok = MBAR_WAIT_ROLE(bar(BAR_PFULL + 1), (uint32_t)(f & 1), abort_flag, p.status, 26);
+          ok = mbar_wait1(bar(BAR_PFULL + 1), (uint32_t)(f & 1), abort_flag, p.status, 26);
           if (!ok) break;
           tc_fence_after();
-          ok = gemm2(1, n0, j0, f);
-          if (!ok) break;
+          gemm2(1, 0, j0, f);
           tc_commit(bar(BAR_KEMPTY + f % kStages));
           if (item_end && f + 1 < F_end) {
             ok = wait_sfree();
             if (!ok) break;
-            ok = gemm1(1, n1, j1, f + 1);
+            ok = gemm1p(1, n1, f + 1, pre_end);
             if (!ok) break;
           }
           if (f + 2 < F_end) {
             ok = wait_kv(f + 2, false);
             if (!ok) break;
-            ok = gemm1(0, n2, j2, f + 2);
+            ok = gemm1p(0, n2, f + 2, pre_end);
             if (!ok) break;
           }
-          n0 = n1; j0 = j1; n1 = n2; j1 = j2;
-          if (++j2 == T) { j2 = 0; ++n2; }
+          if (++j0 == T) { j0 = 0; ++n0; }
         }
       }
     }
@@ -592,15 +596,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       const int64_t grow = (int64_t)qtile * kTile + row;
       if (kPersist && !kOutF32) {
         // Item-walking variant: the epilogue is part of every item's critical path.  Row sum and all 64 accumulator
-        // columns are loaded with one wait, the accumulator is handed back to the issuer at once, then the bf16
-        // rows go to this warp's swizzled box and out as one tensor copy (see the comments of the general path).
+        // columns are loaded with one wait, then the bf16 rows go to this warp's swizzled box and out as one tensor
+        // copy (see the comments of the general path).
         uint32_t lr = 0, r64[kCols];
         if (kPnq) asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(lr) : "r"(t_o + 128) : "memory");
         TMEM_LD64(t_o + kCols * h, r64);
         tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_OFREE + t));   // GEMM 2 of the next item may overwrite the accumulator
         if (kPnq) l = __uint_as_float(lr);
         const float inv_l = 1.0f / l;
         const uint32_t aBox = sbase + kOffOut + (t * 8 + h * 4 + (row >> 5)) * kOutBoxBytes;
@@ -681,11 +682,6 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
                        ::"l"(&out_map), "r"(kCols * h), "r"(qtile * kTile + (row & ~31)), "r"(bh), "r"(aBox) : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
-      }
-      if (kPersist) {                              // this row's accumulator has been read: GEMM 2 of the next item may overwrite it
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_OFREE + t));
       }
       }
     }
