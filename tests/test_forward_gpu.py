@@ -96,6 +96,19 @@ def test_bf16_output_is_rounded_fp32_output():
     assert torch.equal(o32.to(torch.bfloat16), o16)
 
 
+# The bf16 output leaves through shared-memory boxes of 32 rows and tensor copies that clip at Nq; the fp32 output is
+# stored from registers.  Ragged query counts (a box that ends, or lies entirely, beyond Nq; Nq smaller than a box),
+# several heads (a row written past Nq would land in the next head), and the item-walking variant (last case).
+@pytest.mark.parametrize("B,H,nq,nkv", [(1, 3, 1, 1), (1, 3, 31, 200), (1, 3, 77, 40), (1, 3, 130, 3000), (2, 2, 300, 1000),
+                                        (1, 5, 257, 129), (4, 30, 1100, 300)])
+def test_bf16_output_on_ragged_shapes(B, H, nq, nkv):
+    cfg = si.custom_config("br", B, H, nq, nkv, 91 + nq)
+    q, k, v = si.make_all(cfg)
+    o32 = run_forward(cfg, q, k, v, True, True, f32=True)
+    o16 = run_forward(cfg, q, k, v, True, True, f32=False)
+    assert torch.equal(o32.to(torch.bfloat16), o16)
+
+
 def test_constant_v_gives_exactly_normalized_rows_under_pnq():
     # Proposition 1 on the GPU, no oracle involved: V == 1 -> O == 1 under PNQ, != 1 under the direct placement
     cfg = si.custom_config("c", 1, 2, 256, 1024, 61)
