@@ -10,6 +10,8 @@
 * outlier config (H=24, N=8192): the same quality comparison;
 * row-sum diagnostic (Section 5.3): mean row sum of the quantized materialized probabilities and its split
   by quantization outcome, OCP / UOS / UOS+Hadamard, on three synthetic recipes at N=4096;
+* short key/value sequences (cross-attention shapes): H=37, Nq=16384, 1 .. 96 KV tiles of 128 keys, attention launch
+  only on pre-quantized operands: time and TFLOP/s (up to 48 tiles the launch uses the item-walking variant);
 * quantize: 2^20 .. 2^29 bf16 elements, axis 1 and axis 0, OCP and UOS: GB/s and fraction of the
   measured HBM copy rate.
 
@@ -112,6 +114,31 @@ def main():
                 "upward": float(o[:, 4].mean()), "mean_entropy": float(o[:, 5].mean()),
                 "frac_rows_under_normalized": float((o[:, 0] < 1.0).mean())})
         torch.cuda.empty_cache()
+
+    # short key/value sequences: the attention launch alone (operands quantized once, outside the timed region)
+    doc["short_kv"] = []
+    H, Nq = 37, 16384
+    xq = torch.randn((1, H, Nq, 128), device="cuda").to(torch.bfloat16)
+    out = torch.empty((1, H, Nq, 128), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    for tiles in ((1, 4) if args.quick else (1, 2, 4, 8, 16, 32, 48, 64, 96)):
+        Nkv = 128 * tiles
+        xk = torch.randn((1, H, Nkv, 128), device="cuda").to(torch.bfloat16)
+        xv = torch.randn((1, H, Nkv, 128), device="cuda").to(torch.bfloat16)
+        bufs = []
+        for x, axis, n in ((xq, 1, Nq), (xk, 1, Nkv), (xv, 0, Nkv)):
+            nt = -(-n // 128)
+            c = torch.empty((H, nt, 8192), dtype=torch.uint8, device="cuda")
+            sc = torch.empty((H, nt, 512), dtype=torch.uint8, device="cuda")
+            mx.quantize_mxfp4_batched(x, c, sc, H, n, 128, axis, mx.MODE_UOS, mx.LAYOUT_TILE)
+            bufs += [c, sc]
+        ms = timed(lambda: mx.forward_prequantized(*bufs, out, 1, H, Nq, Nkv, 128, 128 ** -0.5,
+                                                   mx.FLAG_UOS | mx.FLAG_PNQ, status), n=10)
+        assert int(status[0]) == 0
+        doc["short_kv"].append({"H": H, "Nq": Nq, "kv_tiles": tiles, "attn_us": ms * 1e3,
+                                "tflops": 4.0 * H * Nq * Nkv * 128 / ms / 1e9})
+    del xq, out
+    torch.cuda.empty_cache()
 
     exps = (20, 24) if args.quick else range(20, 30)
     for e in exps:
