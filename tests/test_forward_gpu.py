@@ -109,6 +109,17 @@ def test_bf16_output_on_ragged_shapes(B, H, nq, nkv):
     assert torch.equal(o32.to(torch.bfloat16), o16)
 
 
+@pytest.mark.parametrize("uos,pnq", [(True, False), (False, True), (False, False)])
+def test_bf16_output_of_the_other_variants_in_the_item_walking_kernel(uos, pnq):
+    cfg = si.custom_config("bv", 3, 60, 520, 700, 17)         # 900 work items of 6 KV tiles, ragged query tail
+    q, k, v = si.make_all(cfg)
+    o32 = run_forward(cfg, q, k, v, uos, pnq, f32=True)
+    o16 = run_forward(cfg, q, k, v, uos, pnq, f32=False)
+    assert torch.equal(o32.to(torch.bfloat16), o16)
+    sample = si.custom_config("bv1", 1, 2, 520, 700, 17)       # the first two heads against the oracle
+    check(o32[:1, :2], oracle_out(sample, q[:1, :2], k[:1, :2], v[:1, :2], uos, pnq))
+
+
 def test_constant_v_gives_exactly_normalized_rows_under_pnq():
     # Proposition 1 on the GPU, no oracle involved: V == 1 -> O == 1 under PNQ, != 1 under the direct placement
     cfg = si.custom_config("c", 1, 2, 256, 1024, 61)
