@@ -186,7 +186,12 @@ static HostPipe* host_pipe(size_t n_events) {
   HostPipe& hp = g_pipe[dev];
   if (!hp.in && cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   if (!hp.out && cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-  if (!hp.quant && cudaStreamCreateWithFlags(&hp.quant, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (!hp.quant) {
+    // the quantize launches are short and feed the next attention launch: they go first when SMs free up
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&hp.quant, cudaStreamNonBlocking, hi) != cudaSuccess) return nullptr;
+  }
   if (!hp.attn && cudaStreamCreateWithFlags(&hp.attn, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
   while (hp.ev.size() < n_events) {
     cudaEvent_t e;
