@@ -1,28 +1,31 @@
-"""MXAttention forward, step by step as Algorithm 2 states it (test infrastructure only).
+"""MXAttention forward on the CPU, written from the definitions of Algorithm 2 (test infrastructure only).
 
-Per head and per query row (rows are independent; the query tile size never enters):
+What is computed, per head and per query row (rows are independent; the query tile size never
+enters the result):
 
-    Q-hat, K-hat = Q(.) with 32-blocks along the head dimension        (Alg. 2 lines 3-4)
-    V-hat        = Q(.) with 32-blocks along the token axis            (Alg. 2 line 5)
-    for each KV tile j of B_c = 128 keys, ascending:                   (line 8)
-        S      = Q-hat K-hat_j^T * softmax_scale                       (line 9)
-        m_new  = max(m, rowmax S)                                      (line 10)
-        alpha  = exp(m - m_new)                                        (line 11)
-        P~     = exp(S - m_new)            rounded once to fp32        (line 12)
-        P-hat  = Q(P~) with 32-blocks along the key axis               (line 13)
-        l      = alpha l + P-hat 1   (PNQ, Eq. 22)  |  alpha l + P~ 1  (direct, Eq. 12)   (line 14)
-        O~     = alpha O~ + P-hat V-hat_j                              (line 15)
-        m      = m_new                                                 (line 16)
-    O = O~ / l                                                         (line 18)
+  * Q-hat, K-hat: Q and K quantized in 32-blocks along the head dimension, optionally after the
+    fixed Hadamard rotation; V-hat: V quantized in 32-blocks along the token axis (Algorithm 2,
+    the quantization steps before the loop; Section 4.3).
+  * The keys are visited in tiles of B_c = 128, in ascending order.  A tile contributes
+      - its scores  S = Q-hat K-hat_tile^T * softmax_scale,
+      - the new running maximum and the decay  alpha = exp(m_old - m_new)  of the state kept so far
+        (the FlashAttention-2 recurrence of Section 2),
+      - the un-normalized probabilities  P~ = exp(S - m_new), rounded ONCE to fp32 -- the precision
+        in which the quantizer sees them --, and their quantized form  P-hat = Q(P~)  in 32-blocks
+        along the key axis,
+      - the row-sum increment: P-hat 1 under pre-normalization quantization (Eq. 22), P~ 1 under
+        the direct placement (Eq. 12),
+      - the accumulator increment  P-hat V-hat_tile.
+  * O = accumulator / row sum.
 
-The Hadamard rotation of lines 1-2 is optional (`rotate`).  The same scale rule (UOS or the
-OCP floor rule) is used for all four tensors Q, K, V and P~ (Section 4.3; the "MXFP4 (OCP)"
-baseline of Section 5.2).  float64 everywhere except the single fp32 rounding of P~, which is
-the precision in which the quantizer sees the exponentials.
+The same scale rule (UOS, or the OCP floor rule) serves all four tensors Q, K, V and P~
+(Section 4.3; the "MXFP4 (OCP)" baseline of Section 5.2).  float64 everywhere except the single
+fp32 rounding of P~.
 
 Readings: B_c is fixed to 128 and tiles are visited in ascending order (the result depends on
-both, because P-hat depends on the running-max history); key columns beyond Nkv are excluded
-from the row max and contribute P~ = 0; the last V block along tokens is zero-extended.
+both, because P-hat depends on the history of the running maximum); key columns beyond Nkv are
+excluded from the row maximum and contribute P~ = 0; the last V block along tokens is
+zero-extended.
 """
 from __future__ import annotations
 
@@ -35,14 +38,38 @@ B_C = 128
 
 def quantize_qkv(q, k, v, rule, rotate: bool = False):
     """Dequantized Q-hat, K-hat, V-hat (float64) of one head. q [Nq,d], k,v [Nkv,d].
-    rotate: apply the fixed Hadamard rotation to Q and K first (Algorithm 2 lines 1-2)."""
+    rotate: apply the fixed Hadamard rotation x -> x H_d / sqrt(d) to Q and K first (Algorithm 2,
+    the rotation steps; the plain definition, `mxfp4.hadamard_rotate`)."""
     if rotate:
-        q = mxfp4.hadamard_rotate_f32(q)
-        k = mxfp4.hadamard_rotate_f32(k)
+        q = mxfp4.hadamard_rotate(q)
+        k = mxfp4.hadamard_rotate(k)
     qd = mxfp4.quantize_dequantize(q, axis=1, rule=rule)
     kd = mxfp4.quantize_dequantize(k, axis=1, rule=rule)
     vd = mxfp4.quantize_dequantize(v, axis=0, rule=rule)
     return qd, kd, vd
+
+
+def tile_probabilities(s, m_new, width: int, quantizer):
+    """Un-normalized probabilities of one key tile and their quantized form.
+
+    s [nq, width] scores of the tile's valid keys, m_new [nq] the running maximum including this tile.
+    Returns (p_tilde, p_hat), both [nq, B_C]: exp(s - m_new) rounded once to fp32, zero in the columns
+    past `width`; and `quantizer` applied to it in 32-blocks along the key axis (None: the identity)."""
+    nq = s.shape[0]
+    p_tilde = np.zeros((nq, B_C))
+    with np.errstate(under="ignore"):
+        p_tilde[:, :width] = np.exp(s - m_new[:, None]).astype(np.float32)
+    if quantizer is None:
+        return p_tilde, p_tilde
+    codes, e = mxfp4.quantize_blocks(p_tilde.reshape(nq, B_C // mxfp4.BLOCK, mxfp4.BLOCK), quantizer)
+    return p_tilde, mxfp4.dequantize_blocks(codes, e).reshape(nq, B_C)
+
+
+def row_sum_increment(p_tilde, p_hat, pnq: bool):
+    """What a tile adds to the softmax denominator: the quantized probabilities under PNQ (Eq. 22), so
+    that numerator and denominator see the same values; the unquantized ones under the direct placement
+    (Eq. 12)."""
+    return (p_hat if pnq else p_tilde).sum(axis=1)
 
 
 def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True,
@@ -71,33 +98,27 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     nkv = kd.shape[0]
     scale = float(np.float32(softmax_scale))          # the fp32 argument value, used as given
 
+    # state of the online softmax: running maximum, denominator, un-normalized output
     m = np.full(nq, -np.inf)
     l = np.zeros(nq)
     o = np.zeros((nq, d))
     state = {"m": [], "p_hat": [], "p_tilde": []} if return_state else None
 
-    for j0 in range(0, nkv, B_C):
-        j1 = min(j0 + B_C, nkv)
-        w = j1 - j0
-        s = (qd @ kd[j0:j1].T) * scale                                    # line 9
-        m_new = np.maximum(m, s.max(axis=1))                              # line 10
-        alpha = np.exp(m - m_new)                                         # line 11 (exp(-inf) = 0)
-        p_tilde = np.zeros((nq, B_C))
-        with np.errstate(under="ignore"):
-            p_tilde[:, :w] = np.exp(s - m_new[:, None]).astype(np.float32)    # line 12, fp32 once
-        if quantize_p:
-            codes, e = mxfp4.quantize_blocks(p_tilde.reshape(nq, B_C // 32, 32), rule)   # line 13
-            p_hat = mxfp4.dequantize_blocks(codes, e).reshape(nq, B_C)
-        else:
-            p_hat = p_tilde
-        l = alpha * l + (p_hat.sum(axis=1) if pnq else p_tilde.sum(axis=1))   # line 14
-        o = alpha[:, None] * o + p_hat[:, :w] @ vd[j0:j1]                      # line 15
-        m = m_new                                                             # line 16
+    for start in range(0, nkv, B_C):
+        stop = min(start + B_C, nkv)
+        width = stop - start
+        s = (qd @ kd[start:stop].T) * scale
+        m_new = np.maximum(m, s.max(axis=1))
+        alpha = np.exp(m - m_new)                     # decay of the state kept so far; exp(-inf) = 0 on the first tile
+        p_tilde, p_hat = tile_probabilities(s, m_new, width, rule if quantize_p else None)
+        l = alpha * l + row_sum_increment(p_tilde, p_hat, pnq)
+        o = alpha[:, None] * o + p_hat[:, :width] @ vd[start:stop]
+        m = m_new
         if return_state:
             state["m"].append(m.copy())
-            state["p_hat"].append(p_hat[:, :w].copy())
-            state["p_tilde"].append(p_tilde[:, :w].copy())
-    out = o / l[:, None]                                                  # line 18
+            state["p_hat"].append(p_hat[:, :width].copy())
+            state["p_tilde"].append(p_tilde[:, :width].copy())
+    out = o / l[:, None]
     if return_state:
         state["l"] = l
         state["o_tilde"] = o

@@ -43,7 +43,7 @@ class ScaleRule:
 
 
 OCP = ScaleRule("floor", 8.0)    # Eq. 5: floor(log2 M) - 2 == floor(log2(M/8)) + 1 (Appendix G, Eq. 57)
-UOS = ScaleRule("ceil", 7.25)    # Eq. 13 with q* = 29/4 (Theorem 1); Algorithm 1 line 6
+UOS = ScaleRule("ceil", 7.25)    # Eq. 13 with q* = 29/4 (Theorem 1); the exponent step of Algorithm 1
 TFS = ScaleRule("ceil", 6.0)     # Eq. 8
 OAS = ScaleRule("ceil", 7.0)     # Appendix G
 
@@ -82,17 +82,18 @@ def shared_exponent(M: np.ndarray, rule: ScaleRule) -> np.ndarray:
 
 
 def quantize_blocks(x: np.ndarray, rule: ScaleRule):
-    """Algorithm 1 on an array of blocks x[..., 32] (any float dtype, finite values).
+    """Block quantization (Section 2; Algorithm 1 for the UOS rule) of an array of blocks x[..., 32]
+    (any float dtype, finite values): the block maximum fixes the shared exponent by `rule` (an all-zero
+    block gets sigma = 1), every element is divided by sigma = 2^e -- exactly -- and projected onto the
+    E2M1 grid; the sign is carried separately.
 
     Returns (codes uint8 [..., 32] with bit 3 = sign and bits 0-2 = grid index, e int32 [...]).
     """
     x64 = np.asarray(x, dtype=np.float64)
     assert x64.shape[-1] == BLOCK
     mag = np.abs(x64)
-    M = mag.max(axis=-1)                                   # line 1
-    e = shared_exponent(M, rule)                           # lines 2-3 (zero block) and 6-7
-    scaled = np.ldexp(mag, -e[..., None])                  # v / sigma, exact
-    idx = e2m1_index(scaled)                               # line 9
+    e = shared_exponent(mag.max(axis=-1), rule)
+    idx = e2m1_index(np.ldexp(mag, -e[..., None]))
     sign = np.signbit(x64).astype(np.uint8)
     return (sign << 3) | idx, e
 
@@ -164,12 +165,26 @@ def hadamard_matrix(n: int) -> np.ndarray:
     return np.where(pop % 2 == 0, 1.0, -1.0)
 
 
-def hadamard_rotate_f32(x: np.ndarray) -> np.ndarray:
-    """x R_H along the last axis with R_H = H_n / sqrt(n) (Algorithm 2 lines 1-2: the fixed orthogonal
-    Hadamard rotation), evaluated in fp32 the way the quantizer sees it: the fast Walsh-Hadamard
-    butterfly with strides 1, 2, 4, ..., n/2, each stage (a, b) -> (a + b, a - b) in IEEE fp32, then one
-    fp32 multiply by fl32(1/sqrt(n)).  Returns fp32.  (The precision and the stage order are part of
-    the definition because the result feeds a rounding decision.)"""
+def hadamard_rotate(x: np.ndarray) -> np.ndarray:
+    """x R_H along the last axis with R_H = H_n / sqrt(n): the fixed orthogonal Hadamard rotation of
+    Algorithm 2 lines 1-2 (Section 4.3), written as its definition.
+
+    The matrix product runs in float64.  For bf16 inputs every entry of x H_n is a sum of 128 numbers with
+    8-bit significands, which float64 holds exactly (unless the exponents in one row span more than about
+    2^37), so the only roundings are the float64 division by sqrt(n) and ONE rounding to fp32 at the end --
+    fp32 being the precision in which the quantizer sees the rotated values.  Returns fp32."""
+    x64 = np.asarray(x, dtype=np.float64)
+    n = x64.shape[-1]
+    return ((x64 @ hadamard_matrix(n)) / np.sqrt(np.float64(n))).astype(np.float32)
+
+
+def hadamard_rotate_fwht_f32(x: np.ndarray) -> np.ndarray:
+    """SECONDARY check, not the definition: the same rotation evaluated entirely in fp32 in the order the
+    library documents for its kernel -- fast Walsh-Hadamard butterfly with strides 1, 2, 4, ..., n/2, each
+    stage (a, b) -> (a + b, a - b) in IEEE fp32, then one fp32 multiply by fl32(1/sqrt(n)).  It differs from
+    `hadamard_rotate` by fp32 rounding noise (about 1e-7 relative), which moves a quantized code only when a
+    value sits that close to a rounding boundary.  Tests use it to check that the kernel follows its documented
+    evaluation order; parity with the paper's definition is judged against `hadamard_rotate`."""
     y = np.array(x, dtype=np.float32, copy=True)
     n = y.shape[-1]
     assert n & (n - 1) == 0

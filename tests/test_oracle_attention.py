@@ -229,10 +229,63 @@ def test_rotation_brings_the_quantized_output_closer_to_dense_attention_on_outli
 
 def test_rotation_with_identity_quantizer_changes_nothing():
     q, k, v = head(32, 256, 24)
-    rq = mxfp4.hadamard_rotate_f32(q).astype(np.float64); rk = mxfp4.hadamard_rotate_f32(k).astype(np.float64)
+    rq = mxfp4.hadamard_rotate(q).astype(np.float64); rk = mxfp4.hadamard_rotate(k).astype(np.float64)
     a = attention.forward_head(rq, rk, v, SCALE, quantize_inputs=False, quantize_p=False)
     b = attention.dense_attention_head(q, k, v, SCALE)
     assert np.abs(a - b).max() < 1e-5
+
+
+def _scalar_bf16(x: float) -> float:
+    """fp32 -> bf16 round-to-nearest-even by exact arithmetic on the significand (Python ints only)."""
+    if x == 0.0:
+        return 0.0
+    mant, exp = math.frexp(abs(x))                 # |x| = mant * 2^exp, mant in [0.5, 1)
+    scaled = Fraction(mant) * 256                  # 8 significant bits: integer part in [128, 256)
+    lo = int(scaled)
+    rem = scaled - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and lo % 2 == 1):
+        lo += 1
+    return math.copysign(math.ldexp(lo, exp - 8), x)
+
+
+def _scalar_bf16_attention(q, k, v, sc, p_for_gemm, p_for_sum):
+    """The recurrence of Section 2 (Eq. 2-3) in scalar Python; `p_for_gemm` / `p_for_sum` say which version
+    of the exponentials ("bf16" or "fp32") enters the P V product and the row sum."""
+    nq, d = q.shape
+    nkv = k.shape[0]
+    pick = lambda p, kind: _scalar_bf16(p) if kind == "bf16" else p
+    out = []
+    for i in range(nq):
+        m, l, o = -math.inf, 0.0, [0.0] * d
+        for j0 in range(0, nkv, 128):
+            cols = range(j0, min(j0 + 128, nkv))
+            s = [sum(float(q[i, t]) * float(k[c, t]) for t in range(d)) * sc for c in cols]
+            m_new = max(m, max(s))
+            alpha = math.exp(m - m_new) if m > -math.inf else 0.0
+            p32 = [float(np.float32(math.exp(x - m_new))) for x in s]
+            l = alpha * l + sum(pick(p, p_for_sum) for p in p32)
+            o = [alpha * o[t] + sum(pick(p, p_for_gemm) * float(v[c, t]) for p, c in zip(p32, cols)) for t in range(d)]
+            m = m_new
+        out.append([x / l for x in o])
+    return np.array(out)
+
+
+def test_bf16_variant_against_scalar_python_loops():
+    # What distinguishes the bf16 variant: the exponentials are rounded to bf16 ONLY for the P V product, and the
+    # row sum is taken from the fp32 exponentials.  The scalar restatement with exactly those choices must agree
+    # to rounding-order noise; with either choice swapped it must not.
+    nq, nkv, d = 3, 300, 16
+    q, k, v = head(nq, nkv, 26)
+    q, k, v = q[:, :d].copy(), k[:, :d].copy(), v[:, :d].copy()
+    scale = 1.0 / math.sqrt(d)
+    sc = float(np.float32(scale))
+    got = attention.forward_head_bf16(q, k, v, scale)
+    assert np.abs(_scalar_bf16_attention(q, k, v, sc, "bf16", "fp32") - got).max() < 1e-12
+    assert np.abs(_scalar_bf16_attention(q, k, v, sc, "bf16", "bf16") - got).max() > 1e-6     # row sum from bf16 P
+    assert np.abs(_scalar_bf16_attention(q, k, v, sc, "fp32", "fp32") - got).max() > 1e-6     # P not rounded at all
+    # the scalar rounding helper and the oracle's agree, ties included
+    xs = np.array([1.0, 1.00390625, 1.01171875, -3.0, 0.1, 1e-20, 3.3895313892515355e+38, 1.0000001], np.float32)
+    assert [float(t) for t in attention._round_to_bf16(xs)] == [_scalar_bf16(float(t)) for t in xs]
 
 
 def test_bf16_variant_oracle_is_dense_attention_up_to_bf16_rounding_of_p():
