@@ -20,12 +20,15 @@ def run_forward(cfg, q, k, v, uos, pnq, f32=True, rotate=False):
     dq, dk, dv = util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v)
     flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | (mx.FLAG_OUT_FP32 if f32 else 0) | \
             (mx.FLAG_HADAMARD if rotate else 0)
-    out = torch.full((cfg.B, cfg.H, cfg.Nq, cfg.d), float("nan"), dtype=torch.float32 if f32 else torch.bfloat16, device="cuda")
-    ws = torch.empty(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), dtype=torch.uint8, device="cuda")
+    # output and workspace sit between canary bands: a write outside either fails the test
+    g_out = util.guarded((cfg.B, cfg.H, cfg.Nq, cfg.d), torch.float32 if f32 else torch.bfloat16, float("nan"))
+    g_ws = util.guarded(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), torch.uint8)
+    out, ws = g_out.t, g_ws.t
     mx.forward_ws(dq, dk, dv, out, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, flags, ws)
     assert mx.device_status(ws) == 0
     assert mx.last_launch_count() == 4
-    return out
+    g_out.check(); g_ws.check()
+    return out.clone()
 
 
 def oracle_out(cfg, q, k, v, uos, pnq, rotate=False):
@@ -224,3 +227,29 @@ def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
     check(run_forward(cfg, q, k, v, True, True), oracle_out(cfg, q, k, v, True, True))
     with pytest.raises(mx.MxAttnError):
         mx.selftest_bounded_wait(status, 0)
+
+
+@pytest.mark.parametrize("uos,pnq", [(True, True), (False, False)])
+def test_registered_workspace_entry_point(uos, pnq):
+    """The two-call form of the interface: mxattn_set_workspace registers caller-owned scratch, mxattn_forward (the
+    signature without a workspace argument) uses it.  Compared with the oracle like every other forward."""
+    import paper_2607_24377_b200 as mx
+    cfg = si.custom_config("reg", 1, 3, 300, 1000, 71)
+    q, k, v = si.make_all(cfg)
+    dq, dk, dv = util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v)
+    g_out = util.guarded((cfg.B, cfg.H, cfg.Nq, cfg.d), torch.float32, float("nan"))
+    g_ws = util.guarded(mx.forward_workspace_bytes(cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d), torch.uint8)
+    flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | mx.FLAG_OUT_FP32
+    mx.set_workspace(g_ws.t)
+    try:
+        mx.forward(dq, dk, dv, g_out.t, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, flags)
+        assert mx.device_status(g_ws.t) == 0 and mx.last_launch_count() == 4
+        g_out.check(); g_ws.check()
+        check(g_out.t, oracle_out(cfg, q, k, v, uos, pnq))
+        # a registered workspace that is too small is refused before anything is launched
+        mx.set_workspace(g_ws.t, nbytes=1024)
+        with pytest.raises(mx.MxAttnError) as ei:
+            mx.forward(dq, dk, dv, g_out.t, cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d, cfg.softmax_scale, flags)
+        assert ei.value.code == -4
+    finally:
+        mx.set_workspace(None)

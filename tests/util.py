@@ -71,3 +71,34 @@ def decode_tile_axis1(tile_codes: np.ndarray, tile_scales: np.ndarray) -> np.nda
         e = tile_scales[tile_scale_offset(r, c)].astype(np.int32) - 127
         out[:, 32 * c:32 * c + 32] = np.ldexp(val, e[:, None])
     return out
+
+
+# ------------------------------------------------------------------------------------------------
+# Canary words around device buffers.  Every buffer a kernel writes (outputs, workspaces) can be taken from
+# `guarded()`: the usable region sits between two guard bands filled with a fixed byte, and `check()` verifies after
+# the kernels have run that no guard byte changed -- an out-of-bounds write just before or after the buffer
+# fails the test even where it would not change the compared output.
+GUARD_BYTES = 4096          # a multiple of 256, so the guarded region keeps the allocation's alignment
+GUARD_FILL = 0xC5
+
+
+class Guarded:
+    def __init__(self, shape, dtype, fill=None):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.n = n
+        self.pad = (-n) % 256
+        self.raw = torch.full((GUARD_BYTES + n + self.pad + GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self):
+        torch.cuda.synchronize()
+        front = self.raw[:GUARD_BYTES]
+        back = self.raw[GUARD_BYTES + self.n:]
+        assert bool((front == GUARD_FILL).all()), "a kernel wrote in front of its buffer"
+        assert bool((back == GUARD_FILL).all()), "a kernel wrote behind its buffer"
+
+
+def guarded(shape, dtype, fill=None) -> Guarded:
+    return Guarded(tuple(shape) if not isinstance(shape, int) else (shape,), dtype, fill)
