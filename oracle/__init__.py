@@ -9,6 +9,8 @@ Modules
 -------
 ``mxfp4``      E2M1 grid, E8M0 shared-scale rules (OCP floor rule, ceiling family, UOS), block
                quantizer (Section 2 "MXFP4 Block Quantization", Algorithm 1), canonical packing.
+``nvfp4``      the comparison format of Section 5.2: 16-element blocks, E4M3 block scales, one fp32 tensor-level
+               scale (the two-level recipe, every step in IEEE fp32: a reading, the paper only names the format).
 ``attention``  tiled online-softmax forward with direct or pre-normalization placement of the
                P-tilde quantizer (Section 2 recurrence, Eq. 12, Eq. 22, Algorithm 2), and the
                float64 dense softmax attention.

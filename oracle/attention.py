@@ -31,18 +31,42 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import mxfp4
+from . import mxfp4, nvfp4
 
 B_C = 128
 
 
-def quantize_qkv(q, k, v, rule, rotate: bool = False):
+def _mxfp4_tile_quantizer(rule):
+    """P~ [nq, B_C] -> Q(P~) with 32-blocks along the key axis under `rule`."""
+    def quantize(p_tilde):
+        nq = p_tilde.shape[0]
+        codes, e = mxfp4.quantize_blocks(p_tilde.reshape(nq, B_C // mxfp4.BLOCK, mxfp4.BLOCK), rule)
+        return mxfp4.dequantize_blocks(codes, e).reshape(nq, B_C)
+    return quantize
+
+
+def _nvfp4_tile_quantizer(p_tilde):
+    """P~ [nq, B_C] -> NVFP4(P~) with 16-blocks along the key axis.  The tensor-level maximum of P~ is known
+    without looking at the data: exp(S - m_new) <= 1, with equality in every row once a tile holds the row
+    maximum; so the tensor scale is the constant 1 / 2688 (a reading: the paper does not say how its NVFP4
+    baseline scales the softmax tile)."""
+    nq = p_tilde.shape[0]
+    codes, sc, s_t = nvfp4.quantize_blocks(p_tilde.reshape(nq, B_C // nvfp4.BLOCK, nvfp4.BLOCK), 1.0)
+    return nvfp4.dequantize_blocks(codes, sc, np.broadcast_to(s_t, sc.shape)).reshape(nq, B_C)
+
+
+def quantize_qkv(q, k, v, rule, rotate: bool = False, fmt: str = "mxfp4"):
     """Dequantized Q-hat, K-hat, V-hat (float64) of one head. q [Nq,d], k,v [Nkv,d].
     rotate: apply the fixed Hadamard rotation x -> x H_d / sqrt(d) to Q and K first (Algorithm 2,
-    the rotation steps; the plain definition, `mxfp4.hadamard_rotate`)."""
+    the rotation steps; the plain definition, `mxfp4.hadamard_rotate`).
+    fmt "nvfp4": the comparison format of Section 5.2 instead of MXFP4 (16-blocks, E4M3 block scales, one
+    tensor-level scale per matrix of the head; `rule` is not used)."""
     if rotate:
         q = mxfp4.hadamard_rotate(q)
         k = mxfp4.hadamard_rotate(k)
+    if fmt == "nvfp4":
+        return (nvfp4.quantize_dequantize(q, axis=1), nvfp4.quantize_dequantize(k, axis=1),
+                nvfp4.quantize_dequantize(v, axis=0))
     qd = mxfp4.quantize_dequantize(q, axis=1, rule=rule)
     kd = mxfp4.quantize_dequantize(k, axis=1, rule=rule)
     vd = mxfp4.quantize_dequantize(v, axis=0, rule=rule)
@@ -54,15 +78,15 @@ def tile_probabilities(s, m_new, width: int, quantizer):
 
     s [nq, width] scores of the tile's valid keys, m_new [nq] the running maximum including this tile.
     Returns (p_tilde, p_hat), both [nq, B_C]: exp(s - m_new) rounded once to fp32, zero in the columns
-    past `width`; and `quantizer` applied to it in 32-blocks along the key axis (None: the identity)."""
+    past `width`; and `quantizer` (a map [nq, B_C] -> [nq, B_C] that quantizes in blocks along the key axis;
+    None: the identity) applied to it."""
     nq = s.shape[0]
     p_tilde = np.zeros((nq, B_C))
     with np.errstate(under="ignore"):
         p_tilde[:, :width] = np.exp(s - m_new[:, None]).astype(np.float32)
     if quantizer is None:
         return p_tilde, p_tilde
-    codes, e = mxfp4.quantize_blocks(p_tilde.reshape(nq, B_C // mxfp4.BLOCK, mxfp4.BLOCK), quantizer)
-    return p_tilde, mxfp4.dequantize_blocks(codes, e).reshape(nq, B_C)
+    return p_tilde, quantizer(p_tilde)
 
 
 def row_sum_increment(p_tilde, p_hat, pnq: bool):
@@ -74,8 +98,11 @@ def row_sum_increment(p_tilde, p_hat, pnq: bool):
 
 def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True,
                  rows=None, quantize_inputs: bool = True, quantize_p: bool = True,
-                 return_state: bool = False, rotate: bool = False):
+                 return_state: bool = False, rotate: bool = False, fmt: str = "mxfp4"):
     """Algorithm 2 for one head.
+
+    fmt "nvfp4" runs the same loop with the NVFP4 quantizer in place of MXFP4 for all four tensors (the
+    "NVFP4" baseline of Section 5.2; `uos` is then ignored, `pnq` still chooses where the row sum comes from).
 
     q [Nq,d], k [Nkv,d], v [Nkv,d]: float arrays holding bf16-representable values.
     rows: optional index array of query rows to compute (default all).
@@ -89,7 +116,7 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     if quantize_inputs:
-        qd, kd, vd = quantize_qkv(q, k, v, rule, rotate)
+        qd, kd, vd = quantize_qkv(q, k, v, rule, rotate, fmt)
     else:
         qd, kd, vd = q, k, v
     if rows is not None:
@@ -103,6 +130,7 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     l = np.zeros(nq)
     o = np.zeros((nq, d))
     state = {"m": [], "p_hat": [], "p_tilde": []} if return_state else None
+    tile_quantizer = None if not quantize_p else (_nvfp4_tile_quantizer if fmt == "nvfp4" else _mxfp4_tile_quantizer(rule))
 
     for start in range(0, nkv, B_C):
         stop = min(start + B_C, nkv)
@@ -110,7 +138,7 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
         s = (qd @ kd[start:stop].T) * scale
         m_new = np.maximum(m, s.max(axis=1))
         alpha = np.exp(m - m_new)                     # decay of the state kept so far; exp(-inf) = 0 on the first tile
-        p_tilde, p_hat = tile_probabilities(s, m_new, width, rule if quantize_p else None)
+        p_tilde, p_hat = tile_probabilities(s, m_new, width, tile_quantizer)
         l = alpha * l + row_sum_increment(p_tilde, p_hat, pnq)
         o = alpha[:, None] * o + p_hat[:, :width] @ vd[start:stop]
         m = m_new
@@ -127,14 +155,14 @@ def forward_head(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = Tr
     return out
 
 
-def forward(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True, rotate: bool = False):
+def forward(q, k, v, softmax_scale: float, uos: bool = True, pnq: bool = True, rotate: bool = False, fmt: str = "mxfp4"):
     """All heads. q [B,H,Nq,d], k,v [B,H,Nkv,d] -> O [B,H,Nq,d] float64."""
     q = np.asarray(q)
     B, H = q.shape[:2]
     out = np.empty(q.shape, dtype=np.float64)
     for b in range(B):
         for h in range(H):
-            out[b, h] = forward_head(q[b, h], k[b, h], v[b, h], softmax_scale, uos, pnq, rotate=rotate)
+            out[b, h] = forward_head(q[b, h], k[b, h], v[b, h], softmax_scale, uos, pnq, rotate=rotate, fmt=fmt)
     return out
 
 
