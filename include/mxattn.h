@@ -112,6 +112,36 @@ int mxattn_quantize_mxfp4_qmax(const void* in, void* codes, void* e8m0_scales, i
                                int64_t rows, int64_t cols, int block_axis, float qmax, int layout,
                                void* stream);
 
+/* ---- NVFP4, the comparison format of the paper (named in its Introduction next to MXFP4; Section 5.2, baseline
+ * "NVFP4": Q, K, V and the softmax tile in that format, nothing else changed) -----------------------------------
+ * Elements are E2M1 codes as above; a block is 16 consecutive elements along the block axis with an E4M3 scale
+ * (OCP 8-bit float, 4 exponent bits with bias 7, 3 mantissa bits, subnormals, no infinities, largest value 448 =
+ * code 0x7E; never negative); each matrix of the batch has one fp32 tensor-level scale.  The paper only names the
+ * format; the arithmetic is the usual two-level recipe, every step in IEEE fp32 in this order:
+ *     g   = fl32(2688 / A)      A = tensor_amax[b], the largest magnitude of matrix b (A = 0: g = 1)
+ *     s_T = fl32(1 / g)         -> tensor_scale[b]
+ *     d   = E4M3( fl32(fl32(M * g) * fl32(1/6)) )   M = block maximum; round-to-nearest-even, saturating at 448
+ *     code = sign | E2M1( fl32(|x| * fl32(g / d)) ) (all codes of the block zero when d = 0)
+ * so that x is approximated by value(code) * d * s_T. */
+
+/* Largest magnitude of each of `batch` bf16 matrices in[batch][rows, cols] -> amax[batch] (device fp32).
+ * rows * cols must be a multiple of 8.  One read pass over the input. */
+int mxattn_tensor_amax(const void* in, void* amax, int64_t batch, int64_t rows, int64_t cols, void* stream);
+
+/* NVFP4 quantization of `batch` bf16 matrices with the tensor maxima `tensor_amax` (device fp32 [batch], e.g. from
+ * mxattn_tensor_amax; a caller that wants one scale for the whole batch passes the same value in every entry).
+ * tensor_scale: device fp32 [batch] that receives s_T, or NULL.
+ * Layouts as for mxattn_quantize_mxfp4_batched with twice the scales:
+ *   canonical  block_axis 1: codes [rows, cols/2], scales [rows, cols/16]          (cols % 16 == 0)
+ *              block_axis 0: codes [cols, rows_pad/2], scales [cols, rows_pad/16]  (transposed; rows_pad = 128*ceil(rows/128);
+ *                            padding blocks have code 0 and scale code 0)
+ *   tile       (cols == 128) codes [ceil(rows/128)][8192] exactly as for MXFP4; scales [ceil(rows/128)][1024]: two
+ *              scale-factor atoms of 512 bytes, atom a = blocks 4a..4a+3 (64 elements); inside an atom the byte of
+ *              (row r, block c mod 4) sits at (r % 32)*16 + (r / 32)*4 + (c mod 4). */
+int mxattn_quantize_nvfp4(const void* in, void* codes, void* e4m3_scales, const void* tensor_amax,
+                          void* tensor_scale, int64_t batch, int64_t rows, int64_t cols, int block_axis,
+                          int layout, void* stream);
+
 /* Bytes of device scratch the forward pass needs for the quantized Q, K, V tile images, their
  * scales and a status word.  0 if the shape is unsupported. */
 size_t mxattn_forward_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);

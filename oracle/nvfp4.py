@@ -1,8 +1,9 @@
 """NVFP4 block quantization on the CPU (test infrastructure only).
 
-NVFP4 is the comparison format of the paper (Introduction: "a finer 16-value block granularity with E4M3
-block scales and an additional tensor-level scale"; Section 5.2, baseline "NVFP4": Q, K, V and the softmax
-tile quantized for the two attention GEMMs, no smoothing).  The paper gives no more than that, so the
+NVFP4 is the comparison format of the paper: its Introduction describes it as E2M1 elements in blocks of 16
+with an E4M3 scale per block plus one more scale per tensor, and the "NVFP4" baseline of Section 5.2 quantizes
+Q, K, V and the softmax tile with it for the two attention GEMMs, without smoothing or extra softmax scaling.
+The paper gives no more than that, so the
 arithmetic below is a READING (listed in the design notes): the widely published two-level recipe,
 
     tensor level   g   = 2688 / A          A = largest magnitude of the tensor, 2688 = 448 * 6

@@ -43,6 +43,8 @@ def lib() -> ctypes.CDLL:
         L.mxattn_quantize_mxfp4.argtypes = [vp, vp, vp, i64, i64, ci, ci, vp]
         L.mxattn_quantize_mxfp4_batched.argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, ci, vp]
         L.mxattn_quantize_mxfp4_qmax.argtypes = [vp, vp, vp, i64, i64, i64, ci, cf, ci, vp]
+        L.mxattn_tensor_amax.argtypes = [vp, vp, i64, i64, i64, vp]
+        L.mxattn_quantize_nvfp4.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
         L.mxattn_forward_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_workspace_bytes.restype = sz
         L.mxattn_set_workspace.argtypes = [vp, sz]
@@ -100,6 +102,15 @@ def quantize_mxfp4_batched(inp, codes, e8m0_scales, batch, rows, cols, block_axi
 def quantize_mxfp4_qmax(inp, codes, e8m0_scales, batch, rows, cols, block_axis, qmax, layout):
     _check(lib().mxattn_quantize_mxfp4_qmax(_ptr(inp), _ptr(codes), _ptr(e8m0_scales), batch, rows, cols,
                                             block_axis, qmax, layout, _stream()), "mxattn_quantize_mxfp4_qmax")
+
+
+def tensor_amax(inp, amax, batch, rows, cols):
+    _check(lib().mxattn_tensor_amax(_ptr(inp), _ptr(amax), batch, rows, cols, _stream()), "mxattn_tensor_amax")
+
+
+def quantize_nvfp4(inp, codes, e4m3_scales, tensor_amax, tensor_scale, batch, rows, cols, block_axis, layout):
+    _check(lib().mxattn_quantize_nvfp4(_ptr(inp), _ptr(codes), _ptr(e4m3_scales), _ptr(tensor_amax), _ptr(tensor_scale),
+                                       batch, rows, cols, block_axis, layout, _stream()), "mxattn_quantize_nvfp4")
 
 
 def forward_workspace_bytes(B, H, Nq, Nkv, d) -> int:

@@ -91,6 +91,9 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, int64_t rows,
                     int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream,
                     uint32_t rule_override = 0xFFFFFFFFu);
+int launch_tensor_amax(const void* in, float* amax, int64_t batch, int64_t rows, int64_t cols, cudaStream_t stream);
+int launch_quantize_nvfp4(const void* in, void* codes, void* scales, const float* amax, float* tensor_scale, int64_t batch,
+                          int64_t rows, int64_t cols, int block_axis, int layout, cudaStream_t stream);
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes,
                    const void* k_scales, const void* v_codes, const void* v_scales, void* o,
                    int B, int H, int64_t Nq, int64_t Nkv, float softmax_scale, unsigned flags,
