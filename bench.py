@@ -52,9 +52,11 @@ class ClockSampler(threading.Thread):
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
+    def __init__(self, gpu_id: str):
+        """gpu_id: what nvidia-smi's -i takes.  The GPU's UUID, not the CUDA ordinal: nvidia-smi numbers the
+        machine's GPUs physically and ignores CUDA_VISIBLE_DEVICES, so an ordinal can name another job's GPU."""
         super().__init__(daemon=True)
-        self.index, self.samples, self._stop_evt, self.proc = index, [], threading.Event(), None
+        self.index, self.samples, self._stop_evt, self.proc = gpu_id, [], threading.Event(), None
 
     def run(self):
         try:
@@ -85,29 +87,88 @@ class ClockSampler(threading.Thread):
             except Exception:
                 continue
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "gpu": self.index}
         # median over the samples taken under load (upper half)
         hot = sorted(sm)[len(sm) // 2:]
-        return {"sm_mhz": float(np.median(hot)), "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": float(np.median(hot)), "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm),
+                "gpu": self.index}
+
+
+def gpu_uuid(torch, local: int) -> str:
+    u = str(torch.cuda.get_device_properties(local).uuid)
+    return u if u.startswith("GPU-") else "GPU-" + u
 
 
 # ----------------------------------------------------------------------------------------------
-def oracle_sample(cfg, heads, rows_per_head):
-    """Times the CPU oracle (as it stands) on sampled query rows of `cfg`; returns (TFLOP/s-equivalent, seconds, desc)."""
+def oracle_sample(cfg, heads, rows_per_head, inputs=None, threads=None):
+    """Times the CPU oracle (as it stands) on sampled query rows of `cfg`; returns (TFLOP/s-equivalent, seconds, desc).
+    inputs: optional {head: (q, k, v)} generated beforehand (then input generation is outside the timed region).
+    threads: limit of the BLAS thread pool the oracle's NumPy calls use (None: whatever the environment gives)."""
     from oracle import attention
-    t0 = time.perf_counter()
+    import contextlib
+    limit = contextlib.nullcontext()
+    if threads is not None:
+        from threadpoolctl import threadpool_limits
+        limit = threadpool_limits(limits=threads)
+    f = lambda a: si.bf16_bits_to_f32(a).astype(np.float64)
     n_rows = 0
-    for h in heads:
-        q, k, v = si.make_head(cfg, 0, h)
-        rng = np.random.default_rng([99, h])
-        rows = np.sort(rng.choice(cfg.Nq, rows_per_head, replace=False))
-        f = lambda a: si.bf16_bits_to_f32(a).astype(np.float64)
-        attention.forward_head(f(q), f(k), f(v), cfg.softmax_scale, True, True, rows=rows)
-        n_rows += rows_per_head
-    dt = time.perf_counter() - t0
+    with limit:
+        t0 = time.perf_counter()
+        for h in heads:
+            q, k, v = inputs[h] if inputs is not None else si.make_head(cfg, 0, h)
+            rng = np.random.default_rng([99, h])
+            rows = np.sort(rng.choice(cfg.Nq, rows_per_head, replace=False))
+            attention.forward_head(f(q), f(k), f(v), cfg.softmax_scale, True, True, rows=rows)
+            n_rows += rows_per_head
+        dt = time.perf_counter() - t0
     flops = 4.0 * n_rows * cfg.Nkv * cfg.d
-    return flops / dt / 1e12, dt, f"{rows_per_head} query rows x all {cfg.Nkv} keys in each of heads {list(heads)} " \
-                                  f"(input generation and K/V quantization of those heads included)"
+    return flops / dt / 1e12, dt, f"{rows_per_head} random query rows x all {cfg.Nkv} keys in each of heads {list(heads)} " \
+                                  f"(quantization of those heads' Q, K, V included" + \
+                                  (")" if inputs is not None else ", input generation too)")
+
+
+def probe_fp4_peak(mx, torch, gpu_id):
+    """Measures what the FP4 tensor pipe of this GPU delivers with the library's own dense block-scaled FP4 GEMM
+    (mxattn_probe_fp4_gemm, the same tcgen05.mma kind::mxf4.block_scale the attention kernel issues), with CUDA events
+    and the SM clock sampled meanwhile.  Two figures: `streaming` -- an 8192^3 GEMM whose operands come from global
+    memory --, and `resident` -- the same instruction stream with its operand ring loaded once (issue rate of the
+    tensor pipe itself).  The roofline's denominator is the larger of the two."""
+    M = N = K = 8192
+    kb = K // 128
+    g = torch.Generator(device="cuda"); g.manual_seed(1)
+    ops = []
+    for rows in (M, N):
+        codes = torch.randint(0, 256, (kb, rows // 128, 8192), dtype=torch.uint8, device="cuda", generator=g)
+        scales = torch.randint(124, 131, (kb, rows // 128, 512), dtype=torch.uint8, device="cuda", generator=g)
+        ops += [codes, scales]
+    c = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    out = {"kernel": "fp4_gemm_probe_kernel (128 x 256 tiles, kind::mxf4.block_scale, M = N = 8192)"}
+    for name, k_steps, resident in (("streaming", kb, False), ("resident", 512, True)):
+        flops = 2.0 * M * N * 128 * k_steps
+        for _ in range(3):
+            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status)
+        torch.cuda.synchronize()
+        sampler = ClockSampler(gpu_id); sampler.start(); time.sleep(0.25)
+        n = 12 if resident else 30
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        evs[0].record()
+        for i in range(n):
+            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status)
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        time.sleep(0.15); sampler.stop()
+        ms = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(n))
+        clk = sampler.summary()
+        out[name] = {"k_steps": k_steps, "launches": n, "ms_best": ms[0], "ms_median": ms[n // 2],
+                     "tflops_best": flops / (ms[0] * 1e-3) / 1e12, "tflops_median": flops / (ms[n // 2] * 1e-3) / 1e12,
+                     "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"]}
+    assert int(status[0].item()) == 0, "a bounded device-side wait expired in the FP4 GEMM probe"
+    best = max(("streaming", "resident"), key=lambda k: out[k]["tflops_median"])
+    out["peak_tflops"] = out[best]["tflops_median"]
+    out["peak_mode"] = best
+    out["peak_sm_mhz"] = out[best]["sm_mhz"]
+    return out
 
 
 def cpu_threads():
@@ -155,6 +216,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true")
+    ap.add_argument("--no-fp4-probe", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     cfg = si.CONFIGS[args.workload]
@@ -223,7 +285,8 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local)
+    gpu_id = gpu_uuid(torch, local)
+    sampler = ClockSampler(gpu_id)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
@@ -246,11 +309,29 @@ def main():
     kern_ms = [float(np.mean([evs[i][a].elapsed_time(evs[i][a + 1]) for i in range(args.steps)])) for a in range(4)]
     attn_ms = kern_ms[3]
     attn_tflops = flops / (attn_ms * 1e-3) / 1e12
-    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    # best and median of the attention launch over at least ten launches (the timed steps plus extra launches)
+    attn_all = [evs[i][3].elapsed_time(evs[i][4]) for i in range(args.steps)]
+    for _ in range(max(0, 10 - args.steps)):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        mx.forward_prequantized(qc, qs, kc, ks, vc, vs, out, B, H, Nq, Nkv, d, scale, flags, status)
+        b.record(); torch.cuda.synchronize()
+        attn_all.append(a.elapsed_time(b))
+    attn_all.sort()
+    attn_stats = {"launches": len(attn_all), "ms_best": attn_all[0], "ms_median": attn_all[len(attn_all) // 2],
+                  "tflops_best": flops / (attn_all[0] * 1e-3) / 1e12,
+                  "tflops_median": flops / (attn_all[len(attn_all) // 2] * 1e-3) / 1e12}
     q_elems = [bh * Nq * d, bh * Nkv * d, bh * Nkv * d]
-    quant = {name: {"ms": kern_ms[i], "GBps": QUANT_BYTES_PER_ELEM * q_elems[i] / (kern_ms[i] * 1e-3) / 1e9,
-                    "frac_of_hbm_peak": QUANT_BYTES_PER_ELEM * q_elems[i] / (kern_ms[i] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-             for i, name in enumerate(("q_axis1", "k_axis1", "v_axis0"))}
+    quant = {}
+    for i, name in enumerate(("q_axis1", "k_axis1", "v_axis0")):
+        gbps = QUANT_BYTES_PER_ELEM * q_elems[i] / (kern_ms[i] * 1e-3) / 1e9
+        # two denominators: the copy rate measured on this machine (a plain copy, so a good kernel can read slightly
+        # above 1) and the nominal 8 TB/s the metric names
+        quant[name] = {"ms": kern_ms[i], "GBps": gbps, "frac_of_measured_copy_rate": gbps / peaks["hbm_gbs"],
+                       "frac_of_nominal_8TBps": gbps / 8000.0}
+    fp4 = None
+    if not args.no_fp4_probe and rank == 0:
+        fp4 = probe_fp4_peak(mx, torch, gpu_id)
 
     # ---- variants of the same kernel (kernel-only, a few launches each) ----
     variants = {}
@@ -275,8 +356,9 @@ def main():
             mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, rot, mx.LAYOUT_TILE)
         b.record(); torch.cuda.synchronize()
         ms = a.elapsed_time(b) / 3
-        variants["quantize_q_with_hadamard"] = {"ms": ms, "GBps": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9,
-                                                "frac_of_hbm_peak": QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        gbps = QUANT_BYTES_PER_ELEM * q_elems[0] / (ms * 1e-3) / 1e9
+        variants["quantize_q_with_hadamard"] = {"ms": ms, "GBps": gbps, "frac_of_measured_copy_rate": gbps / peaks["hbm_gbs"],
+                                                "frac_of_nominal_8TBps": gbps / 8000.0}
         mx.quantize_mxfp4_batched(dq, qc, qs, bh, Nq, d, 1, mx.MODE_UOS, mx.LAYOUT_TILE)       # restore the unrotated Q-hat
         # bf16 variant of this repository's own kernel (no quantization; three re-tiling launches + attention)
         wsb = torch.empty(mx.forward_bf16_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
@@ -335,14 +417,49 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        heads = [0, 1] if Nkv <= 20000 else [0]
-        rows = min(cfg.Nq, 6144)                   # about 10-15 s of oracle time at the wan22 size on a 16-core host
-        tf, dt, desc = oracle_sample(cfg, heads, rows)
-        cpu_baseline = {"value": tf, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc,
-                        "seconds": dt}
+        # the oracle as it stands on sampled rows spread over four heads, once on one thread and once on all host cores
+        heads = sorted(set(int(h) for h in np.linspace(0, H - 1, 4)))
+        rows = min(cfg.Nq, 384 if Nkv > 20000 else 1024)
+        inputs = {h: si.make_head(cfg, 0, h) for h in heads}
+        tf_all, dt_all, desc = oracle_sample(cfg, heads, rows, inputs=inputs)
+        n_all = cpu_threads()
+        tf_one, dt_one, _ = oracle_sample(cfg, heads, rows, inputs=inputs, threads=1)
+        cpu_baseline = {"value": tf_all, "unit": UNIT, "cores": n_all, "kind": "oracle", "sample": desc, "seconds": dt_all,
+                        "single_thread": {"value": tf_one, "unit": UNIT, "cores": 1, "seconds": dt_one},
+                        "host_cpus": os.cpu_count(),
+                        "extrapolated_full_workload_hours": cfg.flops / (tf_all * 1e12) / 3600.0}
 
     clocks = sampler.summary()
     mufu_ceiling = 16 * 512 * 148 * clocks["sm_mhz"] * 1e6 / 1e12 if clocks.get("sm_mhz") else None
+    # Roofline of the dominant kernel.  Denominator: the dense FP4 rate measured just above with the library's own
+    # block-scaled GEMM probe ("of measured"); without the probe, the measured sustained cuBLAS bf16 rate times
+    # the nominal FP4 : bf16 ratio.  The two measurements run at different SM clocks (a saturated tensor pipe is
+    # power-capped, this kernel is not), so the fraction is also given per clock: flops per SM cycle over flops per
+    # SM cycle.  What binds this kernel is not the tensor pipe but the exponential unit (one ex2 per score, 16 per
+    # clock and SM against 64 scores' worth of FP4 flops), hence "bound": "mufu" and the fraction of that ceiling.
+    if fp4:
+        fp4_peak = fp4["peak_tflops"]
+        peak_note = (f"dense FP4 measured in this run: mxattn_probe_fp4_gemm, {fp4['peak_mode']} mode, median of "
+                     f"{fp4[fp4['peak_mode']]['launches']} launches at {fp4['peak_sm_mhz']} MHz (of measured)")
+        per_clock = None
+        if clocks.get("sm_mhz") and fp4.get("peak_sm_mhz"):
+            per_clock = (attn_tflops / clocks["sm_mhz"]) / (fp4_peak / fp4["peak_sm_mhz"])
+    else:
+        fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+        peak_note = (f"no FP4 probe in this run: {peaks['source']} sustained bf16 cuBLAS {peaks['bf16_tflops_sustained']} "
+                     f"x nominal ratio 4 (of {peaks['source']})")
+        per_clock = None
+    roofline = {"bound": "mufu", "kernel": "attention_kernel<uos,pnq>", "achieved": attn_tflops,
+                "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak,
+                "frac_per_sm_clock": per_clock, "achieved_sm_mhz": clocks.get("sm_mhz"),
+                "traffic": ATTN_TRAFFIC_PER_TOKEN_HEAD * Nkv * B * H if Nq == Nkv else None,
+                "traffic_note": "ncu dram bytes of a sweep16384 launch scaled by tokens x heads",
+                "peak_note": peak_note,
+                "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms,
+                # the softmax exponentials bind before the tensor pipe does: 16 ex2 per clock per SM,
+                # one per (query, key) pair, 512 tensor flops per pair
+                "mufu_ceiling_tflops": mufu_ceiling, "frac_of_mufu_ceiling": attn_tflops / mufu_ceiling if mufu_ceiling else None,
+                "ncu_cross_check": "profiles/attention_kernel_sweep16384.txt: sm__pipe_tensor_cycles_active 20.9 %, XU pipe 82 %"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -352,15 +469,9 @@ def main():
                    "sharding": "one full batch per GPU, no collective"},
         "clocks": clocks,
         "e2e": e2e, "gpu_launches": 4 * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "attention_kernel<uos,pnq>", "achieved": attn_tflops,
-                     "peak": fp4_peak, "unit": "TFLOP/s", "frac": attn_tflops / fp4_peak,
-                     "traffic": ATTN_TRAFFIC_PER_TOKEN_HEAD * Nkv * B * H if Nq == Nkv else None,
-                     "traffic_note": "ncu dram bytes of a sweep16384 launch scaled by tokens x heads",
-                     "peak_note": f"dense FP4 = {peaks['source']} sustained bf16 cuBLAS {peaks['bf16_tflops_sustained']} x nominal ratio 4 (of {peaks['source']})",
-                     "frac_of_nominal_9PF": attn_tflops / NOMINAL_FP4_TFLOPS, "launch_ms": attn_ms,
-                     # the softmax exponentials bind before the tensor pipe does: 16 ex2 per clock per SM,
-                     # one per (query, key) pair, 512 tensor flops per pair
-                     "mufu_ceiling_tflops": mufu_ceiling, "frac_of_mufu_ceiling": attn_tflops / mufu_ceiling if mufu_ceiling else None},
+        "roofline": roofline,
+        "fp4_peak_probe": fp4,
+        "attention_launch": attn_stats,
         "cpu_baseline": cpu_baseline,
         "kernels_ms": {"quantize_q": kern_ms[0], "quantize_k": kern_ms[1], "quantize_v": kern_ms[2], "attention": attn_ms},
         "quantize": quant, "variants": variants,

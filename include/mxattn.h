@@ -283,6 +283,22 @@ int mxattn_forward_static(const void* q, const void* k, const void* v, void* o,
                           int B, int H, int64_t Nq, int64_t Nkv, int d,
                           float softmax_scale, unsigned flags, void* stream);
 
+/* Dense block-scaled FP4 GEMM, the measuring stick for the attention kernel's two GEMMs (paper Section 1 names the two
+ * matrix products as the dominant operations of the forward pass; Algorithm 2, the score and the output products):
+ *     C[M, N] = A[M, K] B[N, K]^T      MXFP4 operands, fp32 accumulation, C row-major fp32 (out_fp32 != 0) or bf16.
+ * Operands are MXATTN_LAYOUT_TILE images ordered [K/128][rows/128]: tile (kb, t) holds rows 128 t .. 128 t + 127 and
+ * the K elements 128 kb .. 128 kb + 127 -- what mxattn_quantize_mxfp4_batched(batch = K/128, rows, cols = 128,
+ * block_axis 1, MXATTN_LAYOUT_TILE) writes for an input arranged as [K/128][rows][128].
+ * M % 128 == 0, N % 256 == 0, K % 128 == 0, each at most 16384.
+ * resident == 0: k_steps must equal K/128; an ordinary GEMM whose operand tiles stream through shared memory.
+ * resident != 0: the first min(k_steps, 6) K blocks are loaded once and the k_steps (up to 2^20) multiply steps cycle
+ *   over them, so C = sum over steps i of A_(i mod 6) B_(i mod 6)^T: the same instruction stream without global-memory
+ *   traffic, which measures the issue rate of the FP4 tensor pipe itself.
+ * flops = 2 M N 128 k_steps.  `status`: 4 device ints, zeroed by the caller, non-zero if a bounded wait expired. */
+int mxattn_probe_fp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
+                          void* c, int64_t M, int64_t N, int64_t K, int64_t k_steps, int resident, int out_fp32,
+                          void* status, void* stream);
+
 /* Synchronizes `stream`, then copies the workspace's status word to *host_out (host pointer):
  * 0 = no bounded wait expired since the workspace was last used by a forward. */
 int mxattn_device_status(const void* workspace, int* host_out, void* stream);

@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_host_arena_bytes.argtypes = [ci, ci, i64, i64, ci, cu]
         L.mxattn_forward_host_arena_bytes.restype = sz
         L.mxattn_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
+        L.mxattn_probe_fp4_gemm.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, ci, ci, vp, vp]
         L.mxattn_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
         L.mxattn_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.mxattn_last_launch_count.argtypes = []
@@ -190,6 +191,11 @@ def forward_host(q_host, k_host, v_host, o_host, B, H, Nq, Nkv, d, softmax_scale
                                      o_host.data_ptr(), B, H, Nq, Nkv, d, softmax_scale, flags,
                                      _ptr(arena), arena.numel() * arena.element_size(), _stream()),
            "mxattn_forward_host")
+
+
+def probe_fp4_gemm(a_codes, a_scales, b_codes, b_scales, c, M, N, K, k_steps, resident, out_fp32, status):
+    _check(lib().mxattn_probe_fp4_gemm(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), M, N, K,
+                                       k_steps, int(resident), int(out_fp32), _ptr(status), _stream()), "mxattn_probe_fp4_gemm")
 
 
 def device_status(workspace) -> int:
