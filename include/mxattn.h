@@ -310,6 +310,14 @@ int mxattn_device_status(const void* workspace, int* host_out, void* stream);
  * limit of about two seconds. */
 int mxattn_selftest_bounded_wait(void* status, int64_t limit_cycles, void* stream);
 
+/* Exercises, again without disturbing the GPU, the way the attention kernel's paired softmax warps part company when
+ * one of them gives up: two warps that meet at a named barrier in every key tile (each holds half of a query row's
+ * scores; Algorithm 2's row maximum needs both halves).  Warp 0's wait runs out after `limit_cycles` (code 77 in
+ * status[0]); it leaves a NaN mark in its exchange slots and arrives at the meeting without waiting.  Warp 1, whose
+ * own wait succeeded, is thereby released from the meeting, finds the mark and records code 78 in status[1].
+ * `status`: 4 device ints, zeroed by the caller. */
+int mxattn_selftest_pair_abandon(void* status, int64_t limit_cycles, void* stream);
+
 /* Number of kernel launches the last forward call of this process enqueued (for accounting). */
 int mxattn_last_launch_count(void);
 

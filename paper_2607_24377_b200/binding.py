@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_probe_fp4_gemm.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, ci, ci, vp, vp]
         L.mxattn_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
         L.mxattn_selftest_bounded_wait.argtypes = [vp, i64, vp]
+        L.mxattn_selftest_pair_abandon.argtypes = [vp, i64, vp]
         L.mxattn_last_launch_count.argtypes = []
         L.mxattn_strerror.argtypes = [ci]
         L.mxattn_strerror.restype = ctypes.c_char_p
@@ -206,6 +207,10 @@ def device_status(workspace) -> int:
 
 def selftest_bounded_wait(status, limit_cycles: int):
     _check(lib().mxattn_selftest_bounded_wait(_ptr(status), int(limit_cycles), _stream()), "mxattn_selftest_bounded_wait")
+
+
+def selftest_pair_abandon(status, limit_cycles: int):
+    _check(lib().mxattn_selftest_pair_abandon(_ptr(status), int(limit_cycles), _stream()), "mxattn_selftest_pair_abandon")
 
 
 def last_launch_count() -> int:

@@ -416,12 +416,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     const uint32_t aMaxOwn = sbase + kOffMax + (t * 256 + h * 128 + row) * 4;
     const uint32_t aMaxPartner = sbase + kOffMax + (t * 256 + (h ^ 1) * 128 + row) * 4;
     const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
-    // The two warps of a pair meet at an (unbounded) named barrier in every tile, so they must take the same
-    // decision at every bounded wait before it.  Both always wait on the same mbarrier; they therefore give up
-    // only on their own cycle limit, never because another role of the CTA raised the abort flag (a warp that
-    // saw the flag could leave while its partner, a moment later, finds the barrier complete and goes on to
-    // the pair barrier alone).  Their waits watch a flag that nothing sets, and raise the CTA's flag on expiry.
+    // The two warps of a pair meet at a named barrier in every tile.  A warp whose bounded wait runs out leaves through
+    // pair_abandon: a NaN in its exchange slots and a non-blocking arrival at that barrier, so that its partner -- which
+    // may have found the same mbarrier complete a moment earlier and gone on to the meeting -- is released, reads the
+    // NaN in place of a maximum and leaves the same way.  Their waits watch a flag that nothing sets (they give up on
+    // their own cycle limit only) and raise the CTA's flag on expiry.
     volatile int* const own_limit_only = abort_flag + 1;
+    auto abandon = [&]() { pair_abandon(aMaxOwn, aMaxOwn + 2048u, pair_bar); };
     bool ok = true;
     // Work items of this CTA (exactly one without kPersist).  F0 = tiles of the earlier items: the parities of the
     // barriers that complete once per tile follow F0 + j.  X0 counts the earlier exchanges through the half-row
@@ -434,7 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
 
     for (int j = 0; j < T; ++j) {
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)((F0 + j) & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
-      if (!ok) break;
+      if (!ok) { abandon(); break; }
       tc_fence_after();
       uint32_t sr[kCols];
       TMEM_LD64(t_s, sr);
@@ -473,15 +474,18 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       const float partner_max = lds32f(aMaxPartner + par);
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t or rescales
       // O_t; the probe of that barrier is issued while the partner's maximum is on its way
-      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1));
+      // (a NaN from the partner -- it has given up -- takes the same slow path, and is sorted out there)
+      const bool o_ready = ((j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1))) && (partner_max == partner_max);
       const float m_new = max3(m_run, own_max, partner_max);   // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
-        if (!ok) break;
+        ok = !__any_sync(0xFFFFFFFFu, partner_max != partner_max);
+        if (ok && j > 0)
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
+        if (!ok) { abandon(); break; }
       }
       tc_fence_after();
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
@@ -581,13 +585,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       __syncwarp();
     }
-    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
+    if (ok) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
+      if (!ok) abandon();
+    }
     float l = l_run;
-    if (!kPnq) {                                   // add the partner's half of the row sum
+    if (!kPnq && ok) {                             // add the partner's half of the row sum
       const uint32_t par = (uint32_t)((X0 + T) & 1) * 2048u;
       sts32f(aMaxOwn + par, l_run);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       l = l_run + lds32f(aMaxPartner + par);
+      if (__any_sync(0xFFFFFFFFu, l != l)) { ok = false; abandon(); }      // the partner has given up
     }
     if (ok) {
       tc_fence_after();
@@ -716,7 +724,45 @@ __global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles
   if (done && threadIdx.x == 0) atomicCAS(status, 0, -1);      // must not happen
 }
 
+// Self-test of the way two paired softmax warps part company (pair_abandon): warp 0 waits, with a short limit, on a
+// barrier that nothing arrives on, gives up and abandons the pair; warp 1's own wait succeeds, so it goes on to the
+// pair's meeting, must be released from it by warp 0's parting arrival, must find the NaN mark in place of warp 0's
+// value, and records that (code 78 in status[1]).  Nothing faults; the kernel ends normally.
+__global__ void pair_abandon_selftest_kernel(int* status, long long limit_cycles) {
+  __shared__ uint64_t barriers[2];
+  __shared__ int abort_flag[2];
+  __shared__ float slots[2][2][32];                 // [parity][warp][lane]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&barriers[0]), 1);           // never completes
+    mbar_init(smem_u32(&barriers[1]), 1);           // completes at once
+    abort_flag[0] = abort_flag[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_arrive(smem_u32(&barriers[1]));
+  }
+  __syncthreads();
+  const uint32_t own0 = smem_u32(&slots[0][warp][lane]), own1 = smem_u32(&slots[1][warp][lane]);
+  const uint32_t partner0 = smem_u32(&slots[0][warp ^ 1][lane]);
+  const int pair_bar = 1;
+  const bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&barriers[warp]), 0u, &abort_flag[1], status, 77, limit_cycles, &abort_flag[0]));
+  if (!ok) { pair_abandon(own0, own1, pair_bar); return; }
+  sts32f(own0, 1.0f);
+  asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+  const float partner = lds32f(partner0);
+  if (__any_sync(0xFFFFFFFFu, partner != partner)) {
+    if (lane == 0) atomicCAS(status + 1, 0, 78);
+    pair_abandon(own0, own1, pair_bar);
+  } else if (lane == 0) {
+    atomicCAS(status + 1, 0, -1);                   // must not happen: warp 0 never delivers a value
+  }
+}
+
 }  // namespace fwd
+
+int launch_pair_abandon_selftest(int* status, long long limit_cycles, cudaStream_t stream) {
+  fwd::pair_abandon_selftest_kernel<<<1, 64, 0, stream>>>(status, limit_cycles);
+  return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
+}
 
 int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream_t stream) {
   fwd::bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_cycles);

@@ -23,7 +23,7 @@ constexpr int kThreads = 32 * 6;
 constexpr int kStageBytes = kTileCodeBytes * 3 + kTileScaleBytes * 3;    // A tile, two B tiles, their three scale atoms
 constexpr int kOffBar = kStages * kStageBytes;
 constexpr int kSmemBytes = kOffBar + 256 + 1024;
-constexpr uint32_t kColAcc = 0, kColSFA = 256, kColSFB = 264;           // accumulator 256 columns; 2 slots x 4; 2 slots x 8
+constexpr uint32_t kColAcc = 0, kColSF = 256;    // accumulator 256 columns; then scale-factor slots of 12 columns (A: 4, B: 8), one per stage
 
 struct Params {
   const uint8_t* a_codes; const uint8_t* a_scales;     // [K/128][M/128][8192] / [K/128][M/128][512]
@@ -102,10 +102,15 @@ __global__ void __launch_bounds__(kThreads, 1) fp4_gemm_probe_kernel(const Param
           tc_fence_after();
         }
         const uint32_t st = sbase + s * kStageBytes;
-        const uint32_t sfa = tmem + kColSFA + 4 * (i & 1), sfb = tmem + kColSFB + 8 * (i & 1);
-        tc_cp_sf(sfa, st + 3 * kTileCodeBytes);
-        tc_cp_sf(sfb, st + 3 * kTileCodeBytes + kTileScaleBytes);
-        tc_cp_sf(sfb + 4, st + 3 * kTileCodeBytes + 2 * kTileScaleBytes);
+        // scale factors of the stage: tensor-memory slot s.  Streaming: copied for every step (slot s was last read by
+        // the multiplies of step i - kStages, issued long before).  Resident: copied on the first round only, so that
+        // the loop that is timed consists of multiplies alone.
+        const uint32_t sfa = tmem + kColSF + 12 * s, sfb = sfa + 4;
+        if (i < n_loads) {
+          tc_cp_sf(sfa, st + 3 * kTileCodeBytes);
+          tc_cp_sf(sfb, st + 3 * kTileCodeBytes + kTileScaleBytes);
+          tc_cp_sf(sfb + 4, st + 3 * kTileCodeBytes + 2 * kTileScaleBytes);
+        }
         const uint32_t a = st >> 4, b = (st + kTileCodeBytes) >> 4;
         tc_mma(tmem + kColAcc, desc(a), desc(b), make_idesc(kTileN, 0), sfa, sfb, i > 0 ? 1u : 0u);
         tc_mma(tmem + kColAcc, desc(a + 2), desc(b + 2), make_idesc(kTileN, 1), sfa, sfb, 1u);
