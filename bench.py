@@ -143,28 +143,28 @@ def probe_fp4_peak(mx, torch, gpu_id):
         ops += [codes, scales]
     c = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    out = {"kernel": "fp4_gemm_probe_kernel (128 x 256 tiles, kind::mxf4.block_scale, M = N = 8192)"}
-    for name, k_steps, resident in (("streaming", kb, False), ("resident", 512, True)):
+    out = {"kernel": "fp4_gemm_probe_kernel (128 x tile_n tiles, kind::mxf4.block_scale, M = N = 8192)"}
+    for name, k_steps, resident, tile_n in (("streaming", kb, False, 256), ("resident", 510, True, 256), ("resident_n128", 510, True, 128)):
         flops = 2.0 * M * N * 128 * k_steps
         for _ in range(3):
-            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status)
+            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status, tile_n)
         torch.cuda.synchronize()
         sampler = ClockSampler(gpu_id); sampler.start(); time.sleep(0.25)
         n = 12 if resident else 30
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
         evs[0].record()
         for i in range(n):
-            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status)
+            mx.probe_fp4_gemm(*ops, c, M, N, K, k_steps, resident, False, status, tile_n)
             evs[i + 1].record()
         torch.cuda.synchronize()
         time.sleep(0.15); sampler.stop()
         ms = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(n))
         clk = sampler.summary()
-        out[name] = {"k_steps": k_steps, "launches": n, "ms_best": ms[0], "ms_median": ms[n // 2],
+        out[name] = {"k_steps": k_steps, "tile_n": tile_n, "launches": n, "ms_best": ms[0], "ms_median": ms[n // 2],
                      "tflops_best": flops / (ms[0] * 1e-3) / 1e12, "tflops_median": flops / (ms[n // 2] * 1e-3) / 1e12,
                      "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"]}
     assert int(status[0].item()) == 0, "a bounded device-side wait expired in the FP4 GEMM probe"
-    best = max(("streaming", "resident"), key=lambda k: out[k]["tflops_median"])
+    best = max(("streaming", "resident", "resident_n128"), key=lambda k: out[k]["tflops_median"])
     out["peak_tflops"] = out[best]["tflops_median"]
     out["peak_mode"] = best
     out["peak_sm_mhz"] = out[best]["sm_mhz"]

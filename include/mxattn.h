@@ -289,15 +289,17 @@ int mxattn_forward_static(const void* q, const void* k, const void* v, void* o,
  * Operands are MXATTN_LAYOUT_TILE images ordered [K/128][rows/128]: tile (kb, t) holds rows 128 t .. 128 t + 127 and
  * the K elements 128 kb .. 128 kb + 127 -- what mxattn_quantize_mxfp4_batched(batch = K/128, rows, cols = 128,
  * block_axis 1, MXATTN_LAYOUT_TILE) writes for an input arranged as [K/128][rows][128].
- * M % 128 == 0, N % 256 == 0, K % 128 == 0, each at most 16384.
+ * tile_n: columns of C per CTA, 256 or 128 (the N of the multiply instruction; a CTA always takes 128 rows).
+ * M % 128 == 0, N % tile_n == 0, K % 128 == 0, each at most 16384.
  * resident == 0: k_steps must equal K/128; an ordinary GEMM whose operand tiles stream through shared memory.
- * resident != 0: the first min(k_steps, 6) K blocks are loaded once and the k_steps (up to 2^20) multiply steps cycle
- *   over them, so C = sum over steps i of A_(i mod 6) B_(i mod 6)^T: the same instruction stream without global-memory
- *   traffic, which measures the issue rate of the FP4 tensor pipe itself.
+ * resident != 0: the first min(k_steps, 6) K blocks are loaded once and the k_steps (up to 2^20; beyond 6 a multiple of
+ *   6, with K >= 768) multiply steps cycle over them, so C = sum over steps i of A_(i mod 6) B_(i mod 6)^T: after the
+ *   first round the issuing thread executes multiply instructions only -- no global-memory traffic, no scale copies,
+ *   no barriers --, which measures the rate of the FP4 tensor pipe itself.
  * flops = 2 M N 128 k_steps.  `status`: 4 device ints, zeroed by the caller, non-zero if a bounded wait expired. */
 int mxattn_probe_fp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
                           void* c, int64_t M, int64_t N, int64_t K, int64_t k_steps, int resident, int out_fp32,
-                          void* status, void* stream);
+                          int tile_n, void* status, void* stream);
 
 /* Synchronizes `stream`, then copies the workspace's status word to *host_out (host pointer):
  * 0 = no bounded wait expired since the workspace was last used by a forward. */
@@ -310,13 +312,13 @@ int mxattn_device_status(const void* workspace, int* host_out, void* stream);
  * limit of about two seconds. */
 int mxattn_selftest_bounded_wait(void* status, int64_t limit_cycles, void* stream);
 
-/* Exercises, again without disturbing the GPU, the way the attention kernel's paired softmax warps part company when
- * one of them gives up: two warps that meet at a named barrier in every key tile (each holds half of a query row's
- * scores; Algorithm 2's row maximum needs both halves).  Warp 0's wait runs out after `limit_cycles` (code 77 in
- * status[0]); it leaves a NaN mark in its exchange slots and arrives at the meeting without waiting.  Warp 1, whose
- * own wait succeeded, is thereby released from the meeting, finds the mark and records code 78 in status[1].
- * `status`: 4 device ints, zeroed by the caller. */
-int mxattn_selftest_pair_abandon(void* status, int64_t limit_cycles, void* stream);
+/* Exercises, again without disturbing the GPU, the way the attention kernel's paired softmax warps stay in step when
+ * one of them gives up: two warps meet at a named barrier in every key tile (each holds half of a query row's scores;
+ * the row maximum of Algorithm 2 needs both halves).  Here warp 0's wait runs out after `limit_cycles` (code 77 in
+ * status[0]); from then on it only keeps the pair's remaining appointments, as the attention kernel's warps do.
+ * Warp 1, whose waits all succeed, works through `meetings` (1 .. 100000) of them and records how many it completed
+ * in status[1] -- `meetings` if no warp was left stranded.  `status`: 4 device ints, zeroed by the caller. */
+int mxattn_selftest_pair_abandon(void* status, int64_t limit_cycles, int meetings, void* stream);
 
 /* Number of kernel launches the last forward call of this process enqueued (for accounting). */
 int mxattn_last_launch_count(void);

@@ -62,10 +62,10 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_host_arena_bytes.argtypes = [ci, ci, i64, i64, ci, cu]
         L.mxattn_forward_host_arena_bytes.restype = sz
         L.mxattn_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
-        L.mxattn_probe_fp4_gemm.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, ci, ci, vp, vp]
+        L.mxattn_probe_fp4_gemm.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, ci, ci, ci, vp, vp]
         L.mxattn_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
         L.mxattn_selftest_bounded_wait.argtypes = [vp, i64, vp]
-        L.mxattn_selftest_pair_abandon.argtypes = [vp, i64, vp]
+        L.mxattn_selftest_pair_abandon.argtypes = [vp, i64, ci, vp]
         L.mxattn_last_launch_count.argtypes = []
         L.mxattn_strerror.argtypes = [ci]
         L.mxattn_strerror.restype = ctypes.c_char_p
@@ -194,9 +194,10 @@ def forward_host(q_host, k_host, v_host, o_host, B, H, Nq, Nkv, d, softmax_scale
            "mxattn_forward_host")
 
 
-def probe_fp4_gemm(a_codes, a_scales, b_codes, b_scales, c, M, N, K, k_steps, resident, out_fp32, status):
+def probe_fp4_gemm(a_codes, a_scales, b_codes, b_scales, c, M, N, K, k_steps, resident, out_fp32, status, tile_n=256):
     _check(lib().mxattn_probe_fp4_gemm(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), M, N, K,
-                                       k_steps, int(resident), int(out_fp32), _ptr(status), _stream()), "mxattn_probe_fp4_gemm")
+                                       k_steps, int(resident), int(out_fp32), int(tile_n), _ptr(status), _stream()),
+           "mxattn_probe_fp4_gemm")
 
 
 def device_status(workspace) -> int:
@@ -209,8 +210,9 @@ def selftest_bounded_wait(status, limit_cycles: int):
     _check(lib().mxattn_selftest_bounded_wait(_ptr(status), int(limit_cycles), _stream()), "mxattn_selftest_bounded_wait")
 
 
-def selftest_pair_abandon(status, limit_cycles: int):
-    _check(lib().mxattn_selftest_pair_abandon(_ptr(status), int(limit_cycles), _stream()), "mxattn_selftest_pair_abandon")
+def selftest_pair_abandon(status, limit_cycles: int, meetings: int):
+    _check(lib().mxattn_selftest_pair_abandon(_ptr(status), int(limit_cycles), int(meetings), _stream()),
+           "mxattn_selftest_pair_abandon")
 
 
 def last_launch_count() -> int:

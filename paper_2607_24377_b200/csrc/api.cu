@@ -378,10 +378,10 @@ extern "C" int mxattn_selftest_bounded_wait(void* status, int64_t limit_cycles, 
   return launch_bounded_wait_selftest(static_cast<int*>(status), (long long)limit_cycles, (cudaStream_t)stream);
 }
 
-extern "C" int mxattn_selftest_pair_abandon(void* status, int64_t limit_cycles, void* stream) {
-  if (!status || limit_cycles <= 0 || limit_cycles > 2000000000LL) return MXATTN_EINVAL;
+extern "C" int mxattn_selftest_pair_abandon(void* status, int64_t limit_cycles, int meetings, void* stream) {
+  if (!status || limit_cycles <= 0 || limit_cycles > 2000000000LL || meetings <= 0 || meetings > 100000) return MXATTN_EINVAL;
   if (!aligned16(status)) return MXATTN_EALIGN;
-  return launch_pair_abandon_selftest(static_cast<int*>(status), (long long)limit_cycles, (cudaStream_t)stream);
+  return launch_pair_abandon_selftest(static_cast<int*>(status), (long long)limit_cycles, meetings, (cudaStream_t)stream);
 }
 
 extern "C" int mxattn_last_launch_count(void) { return g_launches; }

@@ -106,7 +106,7 @@ int launch_rowsum_diag(const void* q_codes, const void* q_scales, const void* k_
                        void* out, int B, int H, int64_t Nq, int64_t Nkv, float softmax_scale, uint32_t rule,
                        int* status, cudaStream_t stream);
 int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream_t stream);
-int launch_pair_abandon_selftest(int* status, long long limit_cycles, cudaStream_t stream);
+int launch_pair_abandon_selftest(int* status, long long limit_cycles, int meetings, cudaStream_t stream);
 void count_launch(int n);
 
 }  // namespace mxattn

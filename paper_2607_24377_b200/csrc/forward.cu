@@ -416,13 +416,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     const uint32_t aMaxOwn = sbase + kOffMax + (t * 256 + h * 128 + row) * 4;
     const uint32_t aMaxPartner = sbase + kOffMax + (t * 256 + (h ^ 1) * 128 + row) * 4;
     const int pair_bar = 1 + (warp & 3) + 4 * t;   // named barrier shared with the partner warp (w, w^4)
-    // The two warps of a pair meet at a named barrier in every tile.  A warp whose bounded wait runs out leaves through
-    // pair_abandon: a NaN in its exchange slots and a non-blocking arrival at that barrier, so that its partner -- which
-    // may have found the same mbarrier complete a moment earlier and gone on to the meeting -- is released, reads the
-    // NaN in place of a maximum and leaves the same way.  Their waits watch a flag that nothing sets (they give up on
+    // The two warps of a pair meet at a named barrier in every tile (and once more per item under direct placement).
+    // A warp whose bounded wait has run out therefore does not leave: it stops computing and waiting, but keeps every
+    // remaining appointment with its partner (keep_company below), for this item and all later ones, so that the
+    // partner -- which may have found the same mbarrier complete a moment earlier -- is never left alone at the
+    // barrier.  The hot path carries no check for this.  Their waits watch a flag that nothing sets (they give up on
     // their own cycle limit only) and raise the CTA's flag on expiry.
     volatile int* const own_limit_only = abort_flag + 1;
-    auto abandon = [&]() { pair_abandon(aMaxOwn, aMaxOwn + 2048u, pair_bar); };
     bool ok = true;
     // Work items of this CTA (exactly one without kPersist).  F0 = tiles of the earlier items: the parities of the
     // barriers that complete once per tile follow F0 + j.  X0 counts the earlier exchanges through the half-row
@@ -433,9 +433,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     m_run = -INFINITY;
     l_run = 0.0f;
 
-    for (int j = 0; j < T; ++j) {
+    int j = 0;                                      // after the loop: the first tile whose meeting has not been kept yet
+    if (ok) for (; j < T; ++j) {
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)((F0 + j) & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
-      if (!ok) { abandon(); break; }
+      if (!ok) break;
       tc_fence_after();
       uint32_t sr[kCols];
       TMEM_LD64(t_s, sr);
@@ -474,18 +475,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       const float partner_max = lds32f(aMaxPartner + par);
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t or rescales
       // O_t; the probe of that barrier is issued while the partner's maximum is on its way
-      // (a NaN from the partner -- it has given up -- takes the same slow path, and is sorted out there)
-      const bool o_ready = ((j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1))) && (partner_max == partner_max);
+      const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1));
       const float m_new = max3(m_run, own_max, partner_max);   // line 10
       const bool moved = (m_new != m_run) && (j > 0);
       const float m_old = m_run;
       m_run = m_new;
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
-        ok = !__any_sync(0xFFFFFFFFu, partner_max != partner_max);
-        if (ok && j > 0)
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
-        if (!ok) { abandon(); break; }
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
+        if (!ok) { ++j; break; }                   // this tile's meeting has been kept
       }
       tc_fence_after();
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
@@ -580,22 +578,20 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
     }
 
+    if (!ok) pair_keep_company(pair_bar, T - j);    // gave up (now or in an earlier item): only the meetings are kept
+
     // ---- epilogue: O = O~ / l (line 18) ----
     if (kPersist && !kOutF32) {                    // the previous item's output copy has read this warp's box
       if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
       __syncwarp();
     }
-    if (ok) {
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
-      if (!ok) abandon();
-    }
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((F0 + T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     float l = l_run;
-    if (!kPnq && ok) {                             // add the partner's half of the row sum
+    if (!kPnq) {                                   // add the partner's half of the row sum (a meeting that is always kept)
       const uint32_t par = (uint32_t)((X0 + T) & 1) * 2048u;
       sts32f(aMaxOwn + par, l_run);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       l = l_run + lds32f(aMaxPartner + par);
-      if (__any_sync(0xFFFFFFFFu, l != l)) { ok = false; abandon(); }      // the partner has given up
     }
     if (ok) {
       tc_fence_after();
@@ -695,7 +691,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     }
     F0 += T;
     X0 += T + (kPnq ? 0 : 1);
-    } while (kPersist && ok && (item += (int)gridDim.x) < p.total_items);
+    } while (kPersist && (item += (int)gridDim.x) < p.total_items);     // also after giving up: the meetings go on
   }
 
   // ---- teardown ------------------------------------------------------------------------------
@@ -724,14 +720,15 @@ __global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles
   if (done && threadIdx.x == 0) atomicCAS(status, 0, -1);      // must not happen
 }
 
-// Self-test of the way two paired softmax warps part company (pair_abandon): warp 0 waits, with a short limit, on a
-// barrier that nothing arrives on, gives up and abandons the pair; warp 1's own wait succeeds, so it goes on to the
-// pair's meeting, must be released from it by warp 0's parting arrival, must find the NaN mark in place of warp 0's
-// value, and records that (code 78 in status[1]).  Nothing faults; the kernel ends normally.
-__global__ void pair_abandon_selftest_kernel(int* status, long long limit_cycles) {
+// Self-test of the way two paired softmax warps stay in step when one of them gives up: warp 0 waits, with a short
+// limit, on a barrier that nothing arrives on, gives up (code 77 in status[0]) and from then on only keeps the pair's
+// `meetings` appointments (pair_keep_company, the routine the attention kernel uses); warp 1's own waits succeed, so it
+// works through all its meetings, exchanging a value each time, and must come out of the last one: it then records
+// the number of meetings it completed in status[1].  Nothing faults; the kernel ends normally.
+__global__ void pair_abandon_selftest_kernel(int* status, long long limit_cycles, int meetings) {
   __shared__ uint64_t barriers[2];
   __shared__ int abort_flag[2];
-  __shared__ float slots[2][2][32];                 // [parity][warp][lane]
+  __shared__ float slots[2][32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&barriers[0]), 1);           // never completes
@@ -741,26 +738,23 @@ __global__ void pair_abandon_selftest_kernel(int* status, long long limit_cycles
     mbar_arrive(smem_u32(&barriers[1]));
   }
   __syncthreads();
-  const uint32_t own0 = smem_u32(&slots[0][warp][lane]), own1 = smem_u32(&slots[1][warp][lane]);
-  const uint32_t partner0 = smem_u32(&slots[0][warp ^ 1][lane]);
   const int pair_bar = 1;
-  const bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&barriers[warp]), 0u, &abort_flag[1], status, 77, limit_cycles, &abort_flag[0]));
-  if (!ok) { pair_abandon(own0, own1, pair_bar); return; }
-  sts32f(own0, 1.0f);
-  asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-  const float partner = lds32f(partner0);
-  if (__any_sync(0xFFFFFFFFu, partner != partner)) {
-    if (lane == 0) atomicCAS(status + 1, 0, 78);
-    pair_abandon(own0, own1, pair_bar);
-  } else if (lane == 0) {
-    atomicCAS(status + 1, 0, -1);                   // must not happen: warp 0 never delivers a value
+  int kept = 0;
+  bool ok = true;
+  for (; kept < meetings; ++kept) {
+    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&barriers[warp]), 0u, &abort_flag[1], status, 77, limit_cycles, &abort_flag[0]));
+    if (!ok) break;
+    sts32f(smem_u32(&slots[warp][lane]), (float)kept);
+    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
   }
+  if (!ok) pair_keep_company(pair_bar, meetings - kept);
+  else if (lane == 0) atomicCAS(status + 1, 0, kept);
 }
 
 }  // namespace fwd
 
-int launch_pair_abandon_selftest(int* status, long long limit_cycles, cudaStream_t stream) {
-  fwd::pair_abandon_selftest_kernel<<<1, 64, 0, stream>>>(status, limit_cycles);
+int launch_pair_abandon_selftest(int* status, long long limit_cycles, int meetings, cudaStream_t stream) {
+  fwd::pair_abandon_selftest_kernel<<<1, 64, 0, stream>>>(status, limit_cycles, meetings);
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
 }
 

@@ -7,7 +7,7 @@
 //   * resident mode:  the same instruction stream with the ring loaded once and reused for every K step, which takes
 //                     global memory and L2 out of the picture and measures the issue rate of the tensor pipe itself.
 //
-// One CTA computes a 128 x 256 tile of C.  Roles: warp 0 producer (bulk async copies), warp 1 MMA issuer (one
+// One CTA computes a 128 x 256 (or 128 x 128) tile of C.  Roles: warp 0 producer (bulk async copies), warp 1 MMA issuer (one
 // thread), warps 2-5 epilogue (one thread per row of the tile: tensor memory -> registers -> global memory).
 // Every barrier wait is bounded; on expiry the CTA records a code in `status` and exits normally.
 #include "common.cuh"
@@ -17,7 +17,6 @@ namespace mxattn {
 namespace probe {
 using namespace fwd;
 
-constexpr int kTileN = 256;
 constexpr int kStages = 6;
 constexpr int kThreads = 32 * 6;
 constexpr int kStageBytes = kTileCodeBytes * 3 + kTileScaleBytes * 3;    // A tile, two B tiles, their three scale atoms
@@ -36,8 +35,9 @@ struct Params {
   int resident;                                        // 1: load the first min(k_steps, kStages) blocks once and cycle over them
 };
 
-template <bool kOutF32>
+template <bool kOutF32, int kTileN>
 __global__ void __launch_bounds__(kThreads, 1) fp4_gemm_probe_kernel(const Params p) {
+  constexpr int kBTiles = kTileN / 128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -76,12 +76,12 @@ __global__ void __launch_bounds__(kThreads, 1) fp4_gemm_probe_kernel(const Param
         if (!ok) break;
         const int kb = i % p.k_blocks;
         const uint32_t st = sbase + s * kStageBytes;
-        const int64_t ta = (int64_t)kb * p.m_tiles + mt, tb = (int64_t)kb * p.n_tiles128 + 2 * nt;
-        mbar_expect_tx(bar_full(s), kStageBytes);
+        const int64_t ta = (int64_t)kb * p.m_tiles + mt, tb = (int64_t)kb * p.n_tiles128 + kBTiles * nt;
+        mbar_expect_tx(bar_full(s), (1 + kBTiles) * (kTileCodeBytes + kTileScaleBytes));
         bulk_g2s(st, p.a_codes + ta * kTileCodeBytes, kTileCodeBytes, bar_full(s));
-        bulk_g2s(st + kTileCodeBytes, p.b_codes + tb * kTileCodeBytes, 2 * kTileCodeBytes, bar_full(s));     // tiles 2nt, 2nt+1 are adjacent
+        bulk_g2s(st + kTileCodeBytes, p.b_codes + tb * kTileCodeBytes, kBTiles * kTileCodeBytes, bar_full(s));     // the B tiles of a CTA are adjacent
         bulk_g2s(st + 3 * kTileCodeBytes, p.a_scales + ta * kTileScaleBytes, kTileScaleBytes, bar_full(s));
-        bulk_g2s(st + 3 * kTileCodeBytes + kTileScaleBytes, p.b_scales + tb * kTileScaleBytes, 2 * kTileScaleBytes, bar_full(s));
+        bulk_g2s(st + 3 * kTileCodeBytes + kTileScaleBytes, p.b_scales + tb * kTileScaleBytes, kBTiles * kTileScaleBytes, bar_full(s));
       }
       if (!ok || *abort_flag) {                      // gave up: let the copies in flight land before shared memory is released
         const long long t0 = clock64();
@@ -94,27 +94,38 @@ __global__ void __launch_bounds__(kThreads, 1) fp4_gemm_probe_kernel(const Param
       constexpr uint32_t kDescHi = (512u >> 4) | (1u << 14) | (4u << 29);       // 8-row groups 512 B apart, 64-byte swizzle, K-major
       auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
       bool ok = true;
-      for (int i = 0; i < p.k_steps && ok; ++i) {
+      // first pass over the ring (all steps when streaming): wait for the stage, copy its scale factors into the
+      // stage's tensor-memory slot (slot s was last read by the multiplies of step i - kStages, issued long before),
+      // two multiplies of K = 64
+      for (int i = 0; i < n_loads && ok; ++i) {
         const int s = i % kStages;
-        if (i < n_loads) {
-          ok = mbar_wait(bar_full(s), (uint32_t)((i / kStages) & 1), abort_flag, p.status, 42);
-          if (!ok) break;
-          tc_fence_after();
-        }
+        ok = mbar_wait(bar_full(s), (uint32_t)((i / kStages) & 1), abort_flag, p.status, 42);
+        if (!ok) break;
+        tc_fence_after();
         const uint32_t st = sbase + s * kStageBytes;
-        // scale factors of the stage: tensor-memory slot s.  Streaming: copied for every step (slot s was last read by
-        // the multiplies of step i - kStages, issued long before).  Resident: copied on the first round only, so that
-        // the loop that is timed consists of multiplies alone.
         const uint32_t sfa = tmem + kColSF + 12 * s, sfb = sfa + 4;
-        if (i < n_loads) {
-          tc_cp_sf(sfa, st + 3 * kTileCodeBytes);
-          tc_cp_sf(sfb, st + 3 * kTileCodeBytes + kTileScaleBytes);
-          tc_cp_sf(sfb + 4, st + 3 * kTileCodeBytes + 2 * kTileScaleBytes);
-        }
+        tc_cp_sf(sfa, st + 3 * kTileCodeBytes);
+        tc_cp_sf(sfb, st + 3 * kTileCodeBytes + kTileScaleBytes);
+        if (kBTiles == 2) tc_cp_sf(sfb + 4, st + 3 * kTileCodeBytes + 2 * kTileScaleBytes);
         const uint32_t a = st >> 4, b = (st + kTileCodeBytes) >> 4;
         tc_mma(tmem + kColAcc, desc(a), desc(b), make_idesc(kTileN, 0), sfa, sfb, i > 0 ? 1u : 0u);
         tc_mma(tmem + kColAcc, desc(a + 2), desc(b + 2), make_idesc(kTileN, 1), sfa, sfb, 1u);
         if (!p.resident) tc_commit(bar_empty(s));
+      }
+      // resident mode: everything is in place; the loop that is timed issues multiplies and nothing else
+      if (ok && p.resident && p.k_steps > n_loads) {
+        const int rounds = (p.k_steps - n_loads) / kStages;       // k_steps is a multiple of kStages here (checked on the host)
+        const uint32_t a0 = sbase >> 4, stride = (uint32_t)kStageBytes >> 4;
+#pragma unroll 1
+        for (int r = 0; r < rounds; ++r) {
+#pragma unroll
+          for (int s = 0; s < kStages; ++s) {
+            const uint32_t a = a0 + s * stride, b = a + (kTileCodeBytes >> 4);
+            const uint32_t sfa = tmem + kColSF + 12 * s, sfb = sfa + 4;
+            tc_mma(tmem + kColAcc, desc(a), desc(b), make_idesc(kTileN, 0), sfa, sfb, 1u);
+            tc_mma(tmem + kColAcc, desc(a + 2), desc(b + 2), make_idesc(kTileN, 1), sfa, sfb, 1u);
+          }
+        }
       }
       if (ok) tc_commit(bar_acc);
     }
@@ -164,14 +175,16 @@ __global__ void __launch_bounds__(kThreads, 1) fp4_gemm_probe_kernel(const Param
 
 extern "C" int mxattn_probe_fp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
                                      void* c, int64_t M, int64_t N, int64_t K, int64_t k_steps, int resident, int out_fp32,
-                                     void* status, void* stream) {
+                                     int tile_n, void* status, void* stream) {
   using namespace mxattn;
   using namespace mxattn::probe;
   if (!a_codes || !a_scales || !b_codes || !b_scales || !c || !status) return MXATTN_EINVAL;
   if (M <= 0 || N <= 0 || K <= 0 || k_steps <= 0) return MXATTN_EINVAL;
-  if (M % 128 || N % 256 || K % 128) return MXATTN_EUNSUPPORTED;
+  if (tile_n != 128 && tile_n != 256) return MXATTN_EINVAL;
+  if (M % 128 || N % tile_n || K % 128) return MXATTN_EUNSUPPORTED;
   if (M > 16384 || N > 16384 || K > 16384 || k_steps > (1 << 20)) return MXATTN_EUNSUPPORTED;
   if (!resident && k_steps != K / 128) return MXATTN_EINVAL;
+  if (resident && k_steps > 6 && (k_steps % 6 != 0 || K / 128 < 6)) return MXATTN_EINVAL;
   if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) || !aligned16(c) || !aligned16(status))
     return MXATTN_EALIGN;
   Params p;
@@ -179,9 +192,10 @@ extern "C" int mxattn_probe_fp4_gemm(const void* a_codes, const void* a_scales, 
   p.b_codes = (const uint8_t*)b_codes; p.b_scales = (const uint8_t*)b_scales;
   p.c = c; p.status = (int*)status;
   p.m_tiles = (int)(M / 128); p.n_tiles128 = (int)(N / 128); p.k_blocks = (int)(K / 128); p.k_steps = (int)k_steps; p.resident = resident ? 1 : 0;
-  auto kern = out_fp32 ? fp4_gemm_probe_kernel<true> : fp4_gemm_probe_kernel<false>;
+  auto kern = tile_n == 256 ? (out_fp32 ? fp4_gemm_probe_kernel<true, 256> : fp4_gemm_probe_kernel<false, 256>)
+                            : (out_fp32 ? fp4_gemm_probe_kernel<true, 128> : fp4_gemm_probe_kernel<false, 128>);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return MXATTN_ECUDA;
-  const unsigned grid = (unsigned)(p.m_tiles * (N / kTileN));
+  const unsigned grid = (unsigned)(p.m_tiles * (N / tile_n));
   kern<<<grid, kThreads, kSmemBytes, (cudaStream_t)stream>>>(p);
   count_launch(1);
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;

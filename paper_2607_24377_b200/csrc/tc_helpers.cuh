@@ -124,17 +124,12 @@ __device__ __forceinline__ bool mbar_wait1(uint32_t bar, uint32_t parity, volati
   return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
 
-// Two warps that share query rows (each holds half of the key columns) exchange a float per row through two
-// shared-memory slots (double-buffered) and meet at a 64-thread named barrier.  A warp that stops taking part --
-// a bounded wait of its own ran out, or it met the mark below -- calls pair_abandon exactly once: it leaves a NaN in
-// both of its slots and arrives at the barrier without waiting.  Its partner is thereby released from the next meeting,
-// reads the NaN where a maximum or a row sum should be, and stops too; no warp is ever left waiting at the barrier.
-// (Finite inputs never produce a NaN in these slots.)
-__device__ __forceinline__ void pair_abandon(uint32_t slot_a, uint32_t slot_b, int pair_bar) {
-  sts32f(slot_a, __uint_as_float(0x7FC00000u));
-  sts32f(slot_b, __uint_as_float(0x7FC00000u));
-  __threadfence_block();
-  asm volatile("bar.arrive %0, 64;" ::"r"(pair_bar) : "memory");
+// Two warps that share query rows (each holds half of the key columns) meet at a 64-thread named barrier to exchange
+// a value per row.  A warp that has given up on its own work (a bounded wait ran out) must not simply leave, because
+// its partner may already be on its way to the next meeting; it keeps the remaining `n` appointments and does nothing
+// else.  Kept out of line: it is never executed in a healthy run.
+static __device__ __noinline__ void pair_keep_company(int pair_bar, int n) {
+  for (int i = 0; i < n; ++i) asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
 }
 
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

@@ -229,17 +229,19 @@ def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
         mx.selftest_bounded_wait(status, 0)
 
 
-def test_paired_warps_part_company_without_a_hang():
-    # the two softmax warps of a row pair meet at a named barrier in every tile; if one gives up, the other must be
-    # released and must notice.  A dedicated kernel makes one warp's short-limit wait run out (no fault involved).
+def test_paired_warps_stay_in_step_when_one_gives_up():
+    # the two softmax warps of a row pair meet at a named barrier in every tile; a warp that gives up keeps the
+    # remaining appointments so that its partner is never stranded.  A dedicated kernel makes one warp's short-limit
+    # wait run out (no fault involved) and counts the meetings the healthy warp gets through.
     import paper_2607_24377_b200 as mx
-    status = torch.zeros(4, dtype=torch.int32, device="cuda")
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    mx.selftest_pair_abandon(status, 2_000_000)
-    t1.record(); torch.cuda.synchronize()
-    assert status.tolist()[:2] == [77, 78]
-    assert t0.elapsed_time(t1) < 200.0
+    for meetings in (1, 7, 600):
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        mx.selftest_pair_abandon(status, 2_000_000, meetings)
+        t1.record(); torch.cuda.synchronize()
+        assert status.tolist()[:2] == [77, meetings]
+        assert t0.elapsed_time(t1) < 200.0
     cfg = si.custom_config("after2", 1, 1, 130, 260, 6)
     q, k, v = si.make_all(cfg)
     check(run_forward(cfg, q, k, v, True, False), oracle_out(cfg, q, k, v, True, False))
