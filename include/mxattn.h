@@ -229,6 +229,21 @@ int mxattn_forward_bf16(const void* q, const void* k, const void* v, void* o,
                         float softmax_scale, unsigned flags,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* The paper's comparison baseline "NVFP4" (Section 5.2): the same fused forward pass with Q, K, V and the softmax tile
+ * quantized to NVFP4 (see mxattn_quantize_nvfp4) instead of MXFP4, nothing else changed -- same tiling (KV tiles of
+ * 128 keys in ascending order), same recurrence.  Tensor-level scales: one per head for each of Q, K and V (the
+ * largest magnitude of that head's matrix); for the softmax tile the constant 1/2688, because its largest value is
+ * known to be 1 (readings: the paper does not say how the baseline chooses them).
+ * flags: MXATTN_FLAG_PNQ (row sum from the quantized probabilities, as in MXAttention; without it the direct
+ * placement, which is what the paper's baseline uses) and MXATTN_FLAG_OUT_FP32.  Same tensor layouts as
+ * mxattn_forward.  Enqueues three tensor-maximum launches, three quantize launches and the attention launch.
+ * The workspace (mxattn_forward_nvfp4_workspace_bytes) holds the quantized operands and, at its start, the status word. */
+size_t mxattn_forward_nvfp4_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);
+int mxattn_forward_nvfp4(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int64_t Nq, int64_t Nkv, int d,
+                         float softmax_scale, unsigned flags,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of device memory mxattn_forward_host needs (inputs, output and workspace). */
 size_t mxattn_forward_host_arena_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d, unsigned flags);
 

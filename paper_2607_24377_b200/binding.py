@@ -58,6 +58,9 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_bf16_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_bf16_workspace_bytes.restype = sz
         L.mxattn_forward_bf16.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
+        L.mxattn_forward_nvfp4_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
+        L.mxattn_forward_nvfp4_workspace_bytes.restype = sz
+        L.mxattn_forward_nvfp4.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
         L.mxattn_forward_prequantized.argtypes = [vp] * 7 + [ci, ci, i64, i64, ci, cf, cu, vp, vp]
         L.mxattn_forward_host_arena_bytes.argtypes = [ci, ci, i64, i64, ci, cu]
         L.mxattn_forward_host_arena_bytes.restype = sz
@@ -172,6 +175,16 @@ def forward_bf16(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):
     _check(lib().mxattn_forward_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d, softmax_scale, flags,
                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
            "mxattn_forward_bf16")
+
+
+def forward_nvfp4_workspace_bytes(B, H, Nq, Nkv, d) -> int:
+    return int(lib().mxattn_forward_nvfp4_workspace_bytes(B, H, Nq, Nkv, d))
+
+
+def forward_nvfp4(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace):
+    _check(lib().mxattn_forward_nvfp4(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d, softmax_scale, flags,
+                                      _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                      _stream()), "mxattn_forward_nvfp4")
 
 
 def forward_prequantized(q_codes, q_scales, k_codes, k_scales, v_codes, v_scales, o,

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxattn.so")
-SOURCES = ["quantize.cu", "quantize_nvfp4.cu", "forward.cu", "forward_bf16.cu", "rowsum_diag.cu", "fp4_gemm_probe.cu", "api.cu"]
+SOURCES = ["quantize.cu", "quantize_nvfp4.cu", "forward.cu", "forward_bf16.cu", "forward_nvfp4.cu", "rowsum_diag.cu", "fp4_gemm_probe.cu", "api.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-shared",

@@ -365,6 +365,26 @@ extern "C" int mxattn_forward_bf16(const void* q, const void* k, const void* v, 
                              (cudaStream_t)stream);
 }
 
+extern "C" size_t mxattn_forward_nvfp4_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || d != kHeadDim) return 0;
+  return nvfp4_workspace_bytes(B, H, Nq, Nkv);
+}
+
+extern "C" int mxattn_forward_nvfp4(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq,
+                                    int64_t Nkv, int d, float softmax_scale, unsigned flags, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  if (!q || !k || !v || !o) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (flags & ~(unsigned)(MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32)) return MXATTN_EINVAL;
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < 3.0e38f)) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (!workspace) return MXATTN_EWORKSPACE;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace)) return MXATTN_EALIGN;
+  g_launches = 0;
+  return launch_forward_nvfp4(q, k, v, o, B, H, Nq, Nkv, softmax_scale, flags, workspace, workspace_bytes,
+                              (cudaStream_t)stream);
+}
+
 extern "C" int mxattn_device_status(const void* workspace, int* host_out, void* stream) {
   if (!workspace || !host_out) return MXATTN_EINVAL;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MXATTN_ECUDA;

@@ -102,6 +102,9 @@ size_t forward_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv);
 size_t bf16_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv);
 int launch_forward_bf16(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq, int64_t Nkv,
                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+size_t nvfp4_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv);
+int launch_forward_nvfp4(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq, int64_t Nkv,
+                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, cudaStream_t stream);
 int launch_rowsum_diag(const void* q_codes, const void* q_scales, const void* k_codes, const void* k_scales,
                        void* out, int B, int H, int64_t Nq, int64_t Nkv, float softmax_scale, uint32_t rule,
                        int* status, cudaStream_t stream);
