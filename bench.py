@@ -133,7 +133,7 @@ def probe_fp4_peak(mx, torch, gpu_id):
     and the SM clock sampled meanwhile.  Two figures: `streaming` -- an 8192^3 GEMM whose operands come from global
     memory --, and `resident` -- the same instruction stream with its operand ring loaded once (issue rate of the
     tensor pipe itself).  The roofline's denominator is the larger of the two."""
-    M = N = K = 8192
+    M = N = K = 8192            # (in resident mode 2048 CTAs = 13.8 waves of 148: the partly filled last wave is part of the figure)
     kb = K // 128
     g = torch.Generator(device="cuda"); g.manual_seed(1)
     ops = []
@@ -374,6 +374,21 @@ def main():
                                         "note": "mxattn_forward_bf16: whole call (re-tiling of Q, K, V^T + fused attention)"}
         variants["uos_pnq_step_speedup_over_bf16_same_kernel"] = ms / ms_per_step
         del wsb
+        # the paper's comparison format: the same kernel design on NVFP4 operands (whole call: three tensor maxima,
+        # three quantize launches, attention)
+        wsn = torch.empty(mx.forward_nvfp4_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+        for name, fl in (("nvfp4_direct", 0), ("nvfp4_pnq", mx.FLAG_PNQ)):
+            mx.forward_nvfp4(dq, dk, dv, out, B, H, Nq, Nkv, d, scale, fl, wsn); torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(3):
+                mx.forward_nvfp4(dq, dk, dv, out, B, H, Nq, Nkv, d, scale, fl, wsn)
+            b.record(); torch.cuda.synchronize()
+            assert mx.device_status(wsn) == 0
+            ms = a.elapsed_time(b) / 3
+            variants[name] = {"step_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                              "note": "mxattn_forward_nvfp4: whole call (7 launches)"}
+        del wsn
         # bf16 reference point: NOT a kernel of this repository -- PyTorch's fused SDPA (library flash /
         # cuDNN attention) on the same bf16 tensors.  (The repository's own bf16 variant is `bf16_same_kernel` above.)
         try:

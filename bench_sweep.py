@@ -12,6 +12,9 @@
   by quantization outcome, OCP / UOS / UOS+Hadamard, on three synthetic recipes at N=4096;
 * short key/value sequences (cross-attention shapes): H=37, Nq=16384, 1 .. 96 KV tiles of 128 keys, attention launch
   only on pre-quantized operands: time and TFLOP/s (up to 48 tiles the launch uses the item-walking variant);
+* Q_max study (paper Section 5.4.1 and its table of per-block optima): the ceiling-family boundary swept from 6.00 to
+  8.00 in steps of 0.05 with mxattn_quantize_mxfp4_qmax on synthetic Q, K, V of 40 heads per recipe (the heads stand in
+  for the paper's 40 attention blocks): tensor MSE per point, and the histogram of the per-head optimum;
 * quantize: 2^20 .. 2^29 bf16 elements, axis 1 and axis 0, OCP and UOS: GB/s and fraction of the
   measured HBM copy rate.
 
@@ -82,6 +85,12 @@ def main():
             ms = timed(lambda: mx.forward_ws(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, fl | F32, ws))
             assert mx.device_status(ws) == 0
             rep["variants"][name] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
+        wsn = torch.empty(mx.forward_nvfp4_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+        for name, fl in (("nvfp4_direct", 0), ("nvfp4_pnq", mx.FLAG_PNQ)):      # the paper's comparison format, same kernel design
+            ms = timed(lambda: mx.forward_nvfp4(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, fl | F32, wsn))
+            assert mx.device_status(wsn) == 0
+            rep["variants"][name] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
+        del wsn
         ms = timed(lambda: mx.forward_bf16(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, F32, wsb))
         assert mx.device_status(wsb) == 0
         rep["variants"]["bf16_same_kernel"] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
@@ -140,6 +149,40 @@ def main():
     del xq, out
     torch.cuda.empty_cache()
 
+    # Q_max study: sweep of the ceiling-family boundary (Eq. 7) on synthetic tensors; 40 heads per recipe stand in for the
+    # paper's 40 attention blocks.  Dequantization and the MSE are plain torch operations (a measurement aid).
+    doc["qmax_study"] = []
+    lut = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6, -0., -.5, -1, -1.5, -2, -3, -4, -6], dtype=torch.float32, device="cuda")
+    points = [round(6.0 + 0.05 * i, 2) for i in range(41)]
+    Hq, Nq_ = (8, 1024) if args.quick else (40, 8192)
+    for recipe, seed in (("iid", 21), ("outlier", 22), ("wan", 23), ("hunyuan", 24)):
+        cfg = si.custom_config("qmax_" + recipe, 1, Hq, Nq_, Nq_, seed, recipe)
+        q, k, v = si.make_all(cfg)
+        for tname, bits, axis in (("Q", q, 1), ("K", k, 1), ("V", v, 0)):
+            x = dev(bits)[0]                                            # [H, N, 128] bf16
+            xf = x.float()
+            codes = torch.empty((Hq, Nq_, 64) if axis == 1 else (Hq, 128, Nq_ // 2), dtype=torch.uint8, device="cuda")
+            scales = torch.empty((Hq, Nq_, 4) if axis == 1 else (Hq, 128, Nq_ // 32), dtype=torch.uint8, device="cuda")
+            mse = np.empty((len(points), Hq))
+            for i, qm in enumerate(points):
+                mx.quantize_mxfp4_qmax(x, codes, scales, Hq, Nq_, 128, axis, qm, mx.LAYOUT_CANONICAL)
+                nib = torch.stack([codes & 15, codes >> 4], dim=-1).flatten(-2)              # [..., inner]
+                val = lut[nib.long()] * torch.exp2(scales.float() - 127.0).repeat_interleave(32, dim=-1)
+                if axis == 0:
+                    val = val.transpose(1, 2)                                                # back to [H, N, 128]
+                mse[i] = ((val - xf) ** 2).mean(dim=(1, 2)).double().cpu().numpy()
+            best = np.array(points)[mse.argmin(axis=0)]                                      # per-head optimum
+            curve = mse.mean(axis=1)
+            doc["qmax_study"].append({
+                "recipe": recipe, "tensor": tname, "heads": Hq, "tokens": Nq_,
+                "argmin_of_mean_mse": points[int(curve.argmin())],
+                "mse_at_6.00": float(curve[0]), "mse_at_7.00": float(curve[points.index(7.0)]),
+                "mse_at_7.25": float(curve[points.index(7.25)]), "mse_at_8.00": float(curve[-1]),
+                "pct_heads_optimum_le_7.15": float((best <= 7.151).mean() * 100), "pct_heads_optimum_7.20": float((np.abs(best - 7.20) < 1e-6).mean() * 100),
+                "pct_heads_optimum_7.25": float((np.abs(best - 7.25) < 1e-6).mean() * 100), "pct_heads_optimum_ge_7.30": float((best >= 7.299).mean() * 100),
+                "mean_mse_curve": [float(c) for c in curve]})
+        torch.cuda.empty_cache()
+
     exps = (20, 24) if args.quick else range(20, 30)
     for e in exps:
         n = 1 << e
@@ -156,6 +199,21 @@ def main():
                 gbs = QUANT_BYTES_PER_ELEM * n / ms / 1e6
                 doc["quantize_sweep"].append({"elements": n, "axis": axis, "mode": mname, "ms": ms, "GBps": gbs,
                                               "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
+        # NVFP4 (the comparison format): tensor maximum + quantizer, 2 + 2 + 0.5 + 1/16 bytes per element
+        for axis in (1, 0):
+            batch = max(1, rows // 8192)
+            r = rows // batch
+            rp = -(-r // 128) * 128
+            codes = torch.empty(batch * max(r, rp) * 64, dtype=torch.uint8, device="cuda")
+            scales = torch.empty(batch * max(r, rp) * 8, dtype=torch.uint8, device="cuda")
+            amax = torch.empty(batch, dtype=torch.float32, device="cuda"); ts = torch.empty(batch, dtype=torch.float32, device="cuda")
+            def nv():
+                mx.tensor_amax(x, amax, batch, r, 128)
+                mx.quantize_nvfp4(x, codes, scales, amax, ts, batch, r, 128, axis, mx.LAYOUT_CANONICAL)
+            ms = timed(nv, n=10)
+            gbs = (4.0 + 0.5 + 1.0 / 16.0) * n / ms / 1e6
+            doc["quantize_sweep"].append({"elements": n, "axis": axis, "mode": "nvfp4 (tensor maximum + quantizer)", "ms": ms, "GBps": gbs,
+                                          "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
         del x
     print(json.dumps(doc))
 
