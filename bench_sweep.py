@@ -36,9 +36,61 @@ import synth_inputs as si  # noqa: E402
 from bench import QUANT_BYTES_PER_ELEM, load_peaks  # noqa: E402
 
 
+SOFTMAX_PHASES = ["wait_scores", "load_scores", "maxima", "pair_exchange", "wait_prev_output_product", "block_exponents",
+                  "exponentials_pack", "hand_over", "epilogue_per_item"]
+
+
+def cycle_profile(mx, torch, cfg, dev):
+    """Per-role cycle budget of the UOS + PNQ attention kernel (mxattn_forward_cycle_profile, the kernel compiled with
+    cycle counters): mean SM cycles per key tile in each phase, per role, next to the time of the kernel without counters."""
+    B, H, Nq, Nkv, d = cfg.B, cfg.H, cfg.Nq, cfg.Nkv, cfg.d
+    q, k, v = si.make_all(cfg)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    out = torch.empty((B, H, Nq, d), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(mx.forward_workspace_bytes(B, H, Nq, Nkv, d), dtype=torch.uint8, device="cuda")
+    flags = mx.FLAG_UOS | mx.FLAG_PNQ
+    prof = torch.zeros(mx.forward_cycle_profile_bytes(B, H, Nq, Nkv, d) // 8, dtype=torch.int64, device="cuda")
+
+    def timed(fn, n=5):
+        fn(); torch.cuda.synchronize()
+        ts = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return sorted(ts)[n // 2]
+
+    ms_plain = timed(lambda: mx.forward_ws(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, flags, ws))
+    ref = out.clone()
+    ms_prof = timed(lambda: mx.forward_cycle_profile(dq, dk, dv, out, B, H, Nq, Nkv, d, cfg.softmax_scale, flags, ws, prof))
+    assert mx.device_status(ws) == 0 and torch.equal(out, ref)
+    p = prof.view(-1, 18, 16).cpu().numpy().astype(np.float64)
+    p = p[p[:, 17, 9] > 0]                                    # CTAs that ran (one per SM in the item-walking variant)
+    tiles = p[:, 17, 9][:, None]
+    kv_tiles = -(-Nkv // 128)
+    sm = p[:, :16, :]
+    per_tile = sm[:, :, :8] / np.maximum(sm[:, :, 9:10], 1)   # [cta, warp, phase]
+    rep = {"workload": cfg.name, "H": H, "Nq": Nq, "Nkv": Nkv, "kv_tiles": kv_tiles, "ctas": int(p.shape[0]),
+           "ms_without_counters": ms_plain, "ms_with_counters": ms_prof,
+           "softmax_cycles_per_tile": {SOFTMAX_PHASES[i]: float(per_tile[:, :, i].mean()) for i in range(8)},
+           "softmax_epilogue_cycles_per_item": float((sm[:, :, 8] / np.maximum(sm[:, :, 9] / kv_tiles, 1)).mean()),
+           "issuer_cycles_per_tile": {"loop_total": float((p[:, 17, 8:9] / tiles).mean()),
+                                      "wait_p_hat_tile0": float((p[:, 17, 0:1] / tiles).mean()), "wait_p_hat_tile1": float((p[:, 17, 2:3] / tiles).mean()),
+                                      "wait_q": float((p[:, 17, 5:6] / tiles).mean()), "wait_kv": float((p[:, 17, 6:7] / tiles).mean()),
+                                      "wait_score_buffer": float((p[:, 17, 7:8] / tiles).mean())},
+           "producer_cycles_per_tile": {"loop_total": float((p[:, 16, 8:9] / tiles).mean()), "wait_free_stage": float((p[:, 16, 3:4] / tiles).mean()),
+                                        "wait_free_q_buffer": float((p[:, 16, 5:6] / tiles).mean())}}
+    rep["softmax_cycles_per_tile"]["sum"] = float(per_tile.sum(axis=2).mean())
+    rep["issuer_cycles_per_tile"]["issuing"] = rep["issuer_cycles_per_tile"]["loop_total"] - sum(
+        v for k_, v in rep["issuer_cycles_per_tile"].items() if k_.startswith("wait"))
+    return rep
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--quick", action="store_true", help="smallest sizes only")
+    ap.add_argument("--cycle-profile", default=None, metavar="WORKLOAD",
+                    help="only this: per-role cycle profile of the attention kernel on the named workload (e.g. sweep16384, wan22, wan22_cross)")
     args = ap.parse_args()
     import torch
     import paper_2607_24377_b200 as mx
@@ -95,6 +147,10 @@ def main():
         assert mx.device_status(wsb) == 0
         rep["variants"]["bf16_same_kernel"] = {"step_ms": ms, "step_tflops": cfg.flops / ms / 1e9, "rel_l2_vs_float64_dense": quality()}
         return rep
+
+    if args.cycle_profile:
+        print(json.dumps(cycle_profile(mx, torch, si.CONFIGS[args.cycle_profile], dev)))
+        return
 
     doc = {"peaks": peaks, "attention_sweep": [], "quantize_sweep": []}
     sizes = (4096,) if args.quick else (4096, 16384, 32768, 65536)

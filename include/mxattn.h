@@ -40,9 +40,12 @@ extern "C" {
 typedef enum { MXATTN_MODE_OCP = 0, MXATTN_MODE_UOS = 1 } mxattn_mode;
 /* OR-able into `mode` of the quantizer: first apply the fixed orthogonal Hadamard rotation
  * y = x H_128 / sqrt(128) to every row (paper Algorithm 2, lines 1-2; Section 4.3), then quantize y.
- * H_128 is the Sylvester matrix, H[i][j] = (-1)^popcount(i & j).  The rotation is evaluated in fp32
- * as the fast Walsh-Hadamard butterfly with strides 1, 2, ..., 64, each stage (a, b) -> (a + b, a - b),
- * followed by one multiply by fl32(1/sqrt(128)); there is no rounding to bf16 in between.
+ * H_128 is the Sylvester matrix, H[i][j] = (-1)^popcount(i & j).  There is no rounding to bf16 between the rotation
+ * and the quantizer.  Evaluation order of this library (not part of the paper's definition): fp32 throughout, the
+ * fast Walsh-Hadamard butterfly with strides 1, 2, ..., 64, each stage (a, b) -> (a + b, a - b), then one multiply by
+ * fl32(1/sqrt(128)).  Against the exact product rounded once to fp32 this carries about 1e-7 of relative rounding
+ * noise, which can move a code or a scale byte only where a rotated value sits that close to a rounding boundary
+ * (none in 1.6e7 values of the test recipes).
  * Only block_axis 1 with cols == 128. */
 enum { MXATTN_MODE_HADAMARD = 0x100 };
 
@@ -150,8 +153,8 @@ size_t mxattn_forward_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv, int
  * until all enqueued forwards have finished.  Process-global: not thread-safe. */
 int mxattn_set_workspace(void* dev_ptr, size_t bytes);
 
-/* MXAttention forward (paper Algorithm 2, lines 3-19; the Hadamard rotation of lines 1-2 is not
- * part of this call).  q [B,H,Nq,d], k, v [B,H,Nkv,d] bf16; o [B,H,Nq,d] bf16 (fp32 with
+/* MXAttention forward (paper Algorithm 2: lines 3-19, preceded by the Hadamard rotation of Q and K of lines 1-2
+ * when MXATTN_FLAG_HADAMARD is set).  q [B,H,Nq,d], k, v [B,H,Nkv,d] bf16; o [B,H,Nq,d] bf16 (fp32 with
  * MXATTN_FLAG_OUT_FP32).  d must be 128.  Non-causal, no mask.  softmax_scale > 0 multiplies the
  * quantized product Q-hat K-hat^T (line 9).  KV tiles are 128 keys, visited in ascending order.
  * Enqueues three quantize launches (Q, K along d; V along tokens) and one fused attention
@@ -196,6 +199,26 @@ int mxattn_forward_debug_dump(const void* q, const void* k, const void* v, void*
                               float softmax_scale, unsigned flags,
                               void* workspace, size_t workspace_bytes,
                               void* dump, size_t dump_bytes, void* stream);
+
+/* Performance-analysis aid: mxattn_forward_ws (flags exactly MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ, bf16 output) through
+ * an instantiation of the attention kernel that counts, per role, the SM cycles spent in each phase of the key-tile
+ * loop of Algorithm 2 (the timed kernels are compiled without the counters; reading the cycle counter perturbs the
+ * loop by a few percent).  `profile`: caller-owned device memory of mxattn_forward_cycle_profile_bytes() bytes,
+ * zeroed by the caller, that receives [CTA][warp 0..17][16] int64.  One CTA per work item (two query tiles of one
+ * head), or, for short key/value sequences with more work items than SMs, one CTA per SM (then only the first
+ * #SMs records are written).
+ *   warps 0-15 (softmax): [0] wait for the scores, [1] score load, [2] block and row maxima, [3] exchange with the
+ *     partner warp, [4] wait for the previous output product, [5] block exponents, [6] exponentials + packing
+ *     (+ rescaling), [7] hand-over of P-hat, [8] epilogue, [9] tiles processed;
+ *   warp 16 (copy producer): [3] wait for a free K/V stage, [5] wait for a free Q buffer, [8] whole loop, [9] tiles;
+ *   warp 17 (MMA issuer): [0] / [2] wait for P-hat of query tile 0 / 1, [5] wait for Q, [6] wait for K/V, [7] wait
+ *     for the score buffer, [8] whole loop, [9] tiles. */
+size_t mxattn_forward_cycle_profile_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d);
+int mxattn_forward_cycle_profile(const void* q, const void* k, const void* v, void* o,
+                                 int B, int H, int64_t Nq, int64_t Nkv, int d,
+                                 float softmax_scale, unsigned flags,
+                                 void* workspace, size_t workspace_bytes,
+                                 void* profile, size_t profile_bytes, void* stream);
 
 /* Row-sum diagnostic of MXFP4 probability quantization (paper Section 5.3, figure "Row-sum
  * diagnostics", panels A, B, D).  Per query row: P = softmax(Q-hat K-hat^T * softmax_scale) as if

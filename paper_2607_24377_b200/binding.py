@@ -55,6 +55,9 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_debug_dump_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_debug_dump_bytes.restype = sz
         L.mxattn_forward_debug_dump.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp, sz, vp]
+        L.mxattn_forward_cycle_profile_bytes.argtypes = [ci, ci, i64, i64, ci]
+        L.mxattn_forward_cycle_profile_bytes.restype = sz
+        L.mxattn_forward_cycle_profile.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp, sz, vp]
         L.mxattn_forward_bf16_workspace_bytes.argtypes = [ci, ci, i64, i64, ci]
         L.mxattn_forward_bf16_workspace_bytes.restype = sz
         L.mxattn_forward_bf16.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
@@ -165,6 +168,17 @@ def forward_debug_dump(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, works
                                            _ptr(workspace), workspace.numel() * workspace.element_size(),
                                            _ptr(dump), 0 if dump is None else dump.numel() * dump.element_size(), _stream()),
            "mxattn_forward_debug_dump")
+
+
+def forward_cycle_profile_bytes(B, H, Nq, Nkv, d) -> int:
+    return int(lib().mxattn_forward_cycle_profile_bytes(B, H, Nq, Nkv, d))
+
+
+def forward_cycle_profile(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, profile):
+    _check(lib().mxattn_forward_cycle_profile(_ptr(q), _ptr(k), _ptr(v), _ptr(o), B, H, Nq, Nkv, d, softmax_scale, flags,
+                                              _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                              _ptr(profile), 0 if profile is None else profile.numel() * profile.element_size(), _stream()),
+           "mxattn_forward_cycle_profile")
 
 
 def forward_bf16_workspace_bytes(B, H, Nq, Nkv, d) -> int:

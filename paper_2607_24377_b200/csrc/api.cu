@@ -41,7 +41,7 @@ static bool carve(int B, int H, int64_t Nq, int64_t Nkv, int d, WorkspaceLayout*
 static int forward_ws(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq,
                       int64_t Nkv, int d, float softmax_scale, unsigned flags, void* workspace,
                       size_t workspace_bytes, cudaStream_t stream, void* dump = nullptr,
-                      cudaStream_t qstream = nullptr, cudaEvent_t qdone = nullptr) {
+                      cudaStream_t qstream = nullptr, cudaEvent_t qdone = nullptr, bool profile = false) {
   if (!q || !k || !v || !o) return MXATTN_EINVAL;
   if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
   if (flags & ~(unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ | MXATTN_FLAG_OUT_FP32 | MXATTN_FLAG_HADAMARD)) return MXATTN_EINVAL;
@@ -70,7 +70,7 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
   // lines 6-19
   return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
                         ws + w.v_scales, o, B, H, Nq, Nkv, softmax_scale, flags,
-                        reinterpret_cast<int*>(ws + w.status), stream, dump);
+                        reinterpret_cast<int*>(ws + w.status), stream, dump, profile);
 }
 
 }  // namespace mxattn
@@ -152,6 +152,25 @@ extern "C" int mxattn_forward_debug_dump(const void* q, const void* k, const voi
                     (cudaStream_t)stream, dump);
 }
 
+extern "C" size_t mxattn_forward_cycle_profile_bytes(int B, int H, int64_t Nq, int64_t Nkv, int d) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0 || d != kHeadDim) return 0;
+  return forward_profile_bytes(B, H, Nq, Nkv);
+}
+
+extern "C" int mxattn_forward_cycle_profile(const void* q, const void* k, const void* v, void* o, int B, int H,
+                                            int64_t Nq, int64_t Nkv, int d, float softmax_scale, unsigned flags,
+                                            void* workspace, size_t workspace_bytes, void* profile,
+                                            size_t profile_bytes, void* stream) {
+  if (!profile) return MXATTN_EINVAL;
+  if (flags != (unsigned)(MXATTN_FLAG_UOS | MXATTN_FLAG_PNQ)) return MXATTN_EINVAL;
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nkv <= 0) return MXATTN_EINVAL;
+  if (d != kHeadDim) return MXATTN_EUNSUPPORTED;
+  if (profile_bytes < forward_profile_bytes(B, H, Nq, Nkv)) return MXATTN_EWORKSPACE;
+  if (!aligned16(profile)) return MXATTN_EALIGN;
+  return forward_ws(q, k, v, o, B, H, Nq, Nkv, d, softmax_scale, flags, workspace, workspace_bytes,
+                    (cudaStream_t)stream, profile, nullptr, nullptr, true);
+}
+
 extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_scales, const void* k_codes,
                                            const void* k_scales, const void* v_codes, const void* v_scales,
                                            void* o, int B, int H, int64_t Nq, int64_t Nkv, int d,
@@ -170,10 +189,11 @@ extern "C" int mxattn_forward_prequantized(const void* q_codes, const void* q_sc
 }
 
 // ---------------------------------------------------------------------------------------------
-// Host-buffer form.  Heads are independent, so the call is pipelined head by head over three
-// streams: host->device copies of head h+1 and the device->host copy of head h-1 overlap the
-// kernels of head h (PCIe is full duplex).  The two helper streams and the events are created on
-// first use, once per device, and kept for the life of the process; no device memory is allocated.
+// Host-buffer form.  Heads are independent, so the call is pipelined in stages of one or more heads over five
+// streams -- the caller's and four helper streams (copies in, quantization, a second attention stream, copies out):
+// host->device copies of the next stage and the device->host copy of the previous one overlap the kernels of the
+// current stage (PCIe is full duplex).  The helper streams and the events are created on first use, once per
+// device, and kept for the life of the process; no device memory is allocated.
 struct HostPipe {
   cudaStream_t in = nullptr, quant = nullptr, out = nullptr, attn = nullptr;
   std::vector<cudaEvent_t> ev;

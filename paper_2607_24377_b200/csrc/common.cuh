@@ -97,8 +97,9 @@ int launch_quantize_nvfp4(const void* in, void* codes, void* scales, const float
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes,
                    const void* k_scales, const void* v_codes, const void* v_scales, void* o,
                    int B, int H, int64_t Nq, int64_t Nkv, float softmax_scale, unsigned flags,
-                   int* status, cudaStream_t stream, void* dump = nullptr);
+                   int* status, cudaStream_t stream, void* dump = nullptr, bool profile = false);
 size_t forward_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv);
+size_t forward_profile_bytes(int B, int H, int64_t Nq, int64_t Nkv);
 size_t bf16_workspace_bytes(int B, int H, int64_t Nq, int64_t Nkv);
 int launch_forward_bf16(const void* q, const void* k, const void* v, void* o, int B, int H, int64_t Nq, int64_t Nkv,
                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, cudaStream_t stream);

@@ -128,10 +128,29 @@ struct Params {
 // Waits of the single-thread roles.  In the item-walking variant their loops carry the item bookkeeping as well, and
 // keeping the waits' slow path out of line there shortens the time per tile by 6 %; in the one-item variant the same
 // change measured 3 % slower, so that one keeps the inline form.
-#define MBAR_WAIT_ROLE(...) (kPersist ? mbar_wait1(__VA_ARGS__) : mbar_wait(__VA_ARGS__))
-template <bool kUos, bool kPnq, bool kOutF32, bool kDump, bool kPersist>
+// kProf (cycle profile, never in a timed build): every role accumulates SM cycles per phase of its loop and writes them
+// to p.dump as [CTA][warp 0..17][16] int64 (softmax warps: slots 0-8 = S-full wait, score load, maxima, pair
+// exchange, O-done wait, block exponents, exponentials + pack, hand-over, epilogue; slot 9 = tiles; producer and
+// issuer: slots 0-7 = cycles inside the wait with code c at slot c mod 8, slot 8 = cycles of the whole loop, slot 9 = tiles).
+#define MBAR_WAIT_ROLE(...) (kProf ? prof_wait(__VA_ARGS__) : (kPersist ? mbar_wait1(__VA_ARGS__) : mbar_wait(__VA_ARGS__)))
+#define PROF_MARK(i) do { if (kProf) { const long long prof_now = clock64(); prof_t[i] += prof_now - prof_prev; prof_prev = prof_now; } } while (0)
+constexpr int kProfSlots = 16;
+template <bool kUos, bool kPnq, bool kOutF32, bool kDump, bool kPersist, bool kProf = false>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, const __grid_constant__ CUtensorMap out_map) {
   static_assert(!(kDump && kPersist), "the tile dump is written by the one-item-per-CTA variant only");
+  static_assert(!(kDump && kProf), "the dump buffer holds either the tile dump or the cycle profile");
+  long long prof_t[kProfSlots];
+  long long prof_prev = 0;
+  if (kProf) {
+#pragma unroll
+    for (int i = 0; i < kProfSlots; ++i) prof_t[i] = 0;
+  }
+  auto prof_wait = [&](uint32_t b, uint32_t par, volatile int* af, int* st, int code) {
+    const long long t0 = clock64();
+    const bool r = mbar_wait(b, par, af, st, code);
+    prof_t[code & 7] += clock64() - t0;
+    return r;
+  };
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -184,6 +203,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       int F = 0;                                   // tiles issued so far, over all items of this CTA
       int q_issued = 0;                            // items whose Q tiles were issued
       bool ok = true;
+      if (kProf) prof_prev = clock64();
       for (int n = 0, item = blockIdx.x; (kPersist ? item < p.total_items : n < 1) && ok; ++n, item += gridDim.x) {
         const int bh = item / p.q_pairs, pair = item - bh * p.q_pairs;
         const int qb = kPersist ? (n & 1) : 0;     // Q buffer
@@ -214,6 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
           bulk_g2s(sbase + kOffSFV + s * kTileScaleBytes, p.v_scales + (kv0 + j) * kTileScaleBytes, kTileScaleBytes, bar(BAR_KFULL + s));
         }
       }
+      if (kProf) { prof_t[8] = clock64() - prof_prev; prof_t[9] = F; }
       if (!ok || *abort_flag) {
         // gave up: let copies already in flight land before the CTA's shared memory is released
         const long long t0 = clock64();
@@ -228,6 +249,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
   } else if (warp == kSoftmaxWarps + 1) {
     // =============================== MMA issuer =============================================
     if (lane == 0) {
+      if (kProf) prof_prev = clock64();
       bool ok = MBAR_WAIT_ROLE(bar(BAR_Q), 0, abort_flag, p.status, 21);
       uint32_t sfree_n = 0;      // completed phases of S_FREE consumed so far
       // Descriptor words are loop invariants up to a stage offset: the low word is the shared
@@ -336,7 +358,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
         auto gemm1p = [&](int t, int n, int f, bool edge) {      // n: the item of tile f
           const int qb = n & 1;
           if (t == 0 && edge) {
-            if (!mbar_wait1(bar(BAR_Q + qb), (uint32_t)((n >> 1) & 1), abort_flag, p.status, 21)) return false;
+            if (!MBAR_WAIT_ROLE(bar(BAR_Q + qb), (uint32_t)((n >> 1) & 1), abort_flag, p.status, 21)) return false;
             tc_fence_after();
             tc_cp_sf(tmem + kColSFQ + 0, sbase + kOffSFQ + qb * 2 * kTileScaleBytes);
             tc_cp_sf(tmem + kColSFQ + 4, sbase + kOffSFQ + (qb * 2 + 1) * kTileScaleBytes);
@@ -365,7 +387,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
           const bool item_end = (j0 == T - 1);       // tile f + 1 starts an item
           const bool pre_end = one || (j0 == T - 2); // tile f + 1 ends an item, tile f + 2 starts one
           const int n1 = n0 + (item_end ? 1 : 0), n2 = n1 + (pre_end ? 1 : 0);
-          ok = mbar_wait1(bar(BAR_PFULL + 0), (uint32_t)(f & 1), abort_flag, p.status, 24);
+          ok = MBAR_WAIT_ROLE(bar(BAR_PFULL + 0), (uint32_t)(f & 1), abort_flag, p.status, 24);
           if (!ok) break;
           tc_fence_after();
           gemm2(0, 0, j0, f);
@@ -377,7 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
             ok = gemm1p(1, n1, f + 1, pre_end);
             if (!ok) break;
           }
-          ok = mbar_wait1(bar(BAR_PFULL + 1), (uint32_t)(f & 1), abort_flag, p.status, 26);
+          ok = MBAR_WAIT_ROLE(bar(BAR_PFULL + 1), (uint32_t)(f & 1), abort_flag, p.status, 26);
           if (!ok) break;
           tc_fence_after();
           gemm2(1, 0, j0, f);
@@ -396,6 +418,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
           }
           if (++j0 == T) { j0 = 0; ++n0; }
         }
+      }
+      if (kProf) {
+        prof_t[8] = clock64() - prof_prev;
+        prof_t[9] = kPersist ? (long long)((p.total_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * T : T;
       }
     }
   } else if (warp < kSoftmaxWarps) {
@@ -434,9 +460,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
     l_run = 0.0f;
 
     int j = 0;                                      // after the loop: the first tile whose meeting has not been kept yet
+    if (kProf && F0 == 0) prof_prev = clock64();
     if (ok) for (; j < T; ++j) {
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)((F0 + j) & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
       if (!ok) break;
+      PROF_MARK(0);
       tc_fence_after();
       uint32_t sr[kCols];
       TMEM_LD64(t_s, sr);
@@ -444,6 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_SFREE));  // the score buffer may be overwritten
+      PROF_MARK(1);
 
       if (j == T - 1) {                            // ragged last tile: keys beyond Nkv do not exist
         const int valid = (int)(p.Nkv - (int64_t)j * kTile) - kCols * h;
@@ -470,9 +499,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       for (int b = 1; b < kBlocksPerThread; ++b) own_max = fmaxf(own_max, bmax[b]);
       // half-row maximum -> partner thread (same row, other 64 columns), double-buffered by tile parity
       const uint32_t par = (uint32_t)((X0 + j) & 1) * 2048u;
+      PROF_MARK(2);
       sts32f(aMaxOwn + par, own_max);
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");      // only the two warps that share these rows
       const float partner_max = lds32f(aMaxPartner + par);
+      PROF_MARK(3);
       // GEMM 2 of the previous tile must have read P_t and updated O_t before this tile writes P_t or rescales
       // O_t; the probe of that barrier is issued while the partner's maximum is on its way
       const bool o_ready = (j == 0) || mbar_test(bar(BAR_ODONE + t), (uint32_t)((F0 + j - 1) & 1));
@@ -486,6 +517,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
         if (!ok) { ++j; break; }                   // this tile's meeting has been kept
       }
       tc_fence_after();
+      PROF_MARK(4);
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);     // line 15: O~ <- Diag(alpha) O~
       // alpha = exp(m_old - m_new) (line 11) is exactly 1 for every row of a warp in which no maximum
       // moved, so it is only evaluated on the rescaling path
@@ -517,6 +549,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       }
       // the scale bytes go out before the exponentials, so only the code stores precede the proxy fence
       sts16(aSF, sf_half);
+      PROF_MARK(5);
       uint8_t* dump_tile = nullptr;
       if (kDump && 2 * pair + t < p.q_tiles) {       // image of this (query tile, KV tile): codes, scale atom, m
         dump_tile = p.dump + ((((int64_t)bh * p.q_tiles + 2 * pair + t) * T) + j) * kDumpTileBytes;
@@ -572,10 +605,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       };
       if (rescale) tile_body(std::true_type{}); else tile_body(std::false_type{});
       if (!kPnq) l_run = fmaf(alpha, l_run, l_tile);                         // line 14 (direct)
+      PROF_MARK(6);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
+      PROF_MARK(7);
+      if (kProf) prof_t[9] += 1;
     }
 
     if (!ok) pair_keep_company(pair_bar, T - j);    // gave up (now or in an earlier item): only the meetings are kept
@@ -689,11 +725,17 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
       }
       }
     }
+    PROF_MARK(8);
     F0 += T;
     X0 += T + (kPnq ? 0 : 1);
     } while (kPersist && (item += (int)gridDim.x) < p.total_items);     // also after giving up: the meetings go on
   }
 
+  if (kProf && lane == 0) {
+    long long* dst = reinterpret_cast<long long*>(p.dump) + ((int64_t)blockIdx.x * (kThreads / 32) + warp) * kProfSlots;
+#pragma unroll
+    for (int i = 0; i < kProfSlots; ++i) dst[i] = prof_t[i];
+  }
   // ---- teardown ------------------------------------------------------------------------------
   if (!kOutF32 && warp < kSoftmaxWarps && lane == 0)
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // the output copies have left shared memory
@@ -763,6 +805,11 @@ int launch_bounded_wait_selftest(int* status, long long limit_cycles, cudaStream
   return cudaGetLastError() == cudaSuccess ? MXATTN_OK : MXATTN_ECUDA;
 }
 
+size_t forward_profile_bytes(int B, int H, int64_t Nq, int64_t Nkv) {
+  const int64_t qt = (Nq + kTile - 1) / kTile;
+  return (size_t)((int64_t)B * H * ((qt + 1) / 2) * (fwd::kThreads / 32) * fwd::kProfSlots * 8);     // sized for one CTA per work item
+}
+
 size_t forward_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv) {
   const int64_t qt = (Nq + kTile - 1) / kTile, kt = (Nkv + kTile - 1) / kTile;
   return (size_t)((int64_t)B * H * qt * kt * fwd::kDumpTileBytes + (int64_t)B * H * qt * kTile * 4);
@@ -770,7 +817,7 @@ size_t forward_dump_bytes(int B, int H, int64_t Nq, int64_t Nkv) {
 
 int launch_forward(const void* q_codes, const void* q_scales, const void* k_codes, const void* k_scales,
                    const void* v_codes, const void* v_scales, void* o, int B, int H, int64_t Nq, int64_t Nkv,
-                   float softmax_scale, unsigned flags, int* status, cudaStream_t stream, void* dump) {
+                   float softmax_scale, unsigned flags, int* status, cudaStream_t stream, void* dump, bool profile) {
   using namespace fwd;
   Params p;
   p.q_codes = (const uint8_t*)q_codes; p.q_scales = (const uint8_t*)q_scales;
@@ -796,7 +843,7 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
       return MXATTN_ECUDA;
     n_sm = v;
   }
-  const bool persist = !dump && grid > n_sm && kt <= kPersistMaxTiles;
+  const bool persist = (!dump || profile) && grid > n_sm && kt <= kPersistMaxTiles;
   // Descriptor of the bf16 output as a [B H][Nq][128] tensor with boxes of 32 rows x 64 columns (the epilogue's copies).
   CUtensorMap out_map;
   memset(&out_map, 0, sizeof(out_map));
@@ -826,7 +873,10 @@ int launch_forward(const void* q_codes, const void* q_scales, const void* k_code
   PICK(false, false, false) PICK(false, false, true) PICK(false, true, false) PICK(false, true, true)
   PICK(true, false, false) PICK(true, false, true) PICK(true, true, false) PICK(true, true, true)
 #undef PICK
-  if (dump) {                                     // debug entry point: fp32 output only
+  if (profile) {                                  // cycle profile: the UOS + PNQ, bf16-output kernels with the counters compiled in
+    if (!dump || !uos || !pnq || f32) return MXATTN_EINVAL;
+    kern = persist ? attention_kernel<true, true, false, false, true, true> : attention_kernel<true, true, false, false, false, true>;
+  } else if (dump) {                              // debug entry point: fp32 output only
     if (!f32) return MXATTN_EINVAL;
 #define PICKD(U, P) if (uos == U && pnq == P) kern = attention_kernel<U, P, true, true, false>;
     PICKD(false, false) PICKD(false, true) PICKD(true, false) PICKD(true, true)

@@ -268,12 +268,14 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
     uint8_t* sP = smem + kOffP + t * kTileBytes + h * kHalfBytes;       // this thread's keys are one K half of P
     float* sMax = reinterpret_cast<float*>(smem + kOffMax) + t * 256;
     const int pair_bar = 1 + (warp & 3) + 4 * t;
-    // the two warps of a pair meet at unbounded named barriers, so their bounded waits (always on the same
-    // mbarrier) give up only on their own cycle limit: they watch a flag that nothing sets and raise the CTA's
+    // the two warps of a pair meet at named barriers (twice per tile, twice in the epilogue); a warp whose bounded wait
+    // has run out keeps the remaining appointments (pair_keep_company) so that its partner is never stranded.  Their
+    // waits give up only on their own cycle limit: they watch a flag that nothing sets and raise the CTA's
     volatile int* const own_limit_only = abort_flag + 1;
     bool ok = true;
 
-    for (int j = 0; j < T; ++j) {
+    int j = 0;                                       // after the loop: the first tile whose two meetings have not been kept
+    for (; j < T; ++j) {
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_SFULL + t), (uint32_t)(j & 1), own_limit_only, p.status, 31, kWaitLimitCycles, abort_flag));
       if (!ok) break;
       tc_fence_after();
@@ -313,7 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
       const float nmc = -(m_new * c);
       if (!__all_sync(0xFFFFFFFFu, o_ready)) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((j - 1) & 1), own_limit_only, p.status, 32, kWaitLimitCycles, abort_flag));
-        if (!ok) break;
+        if (!ok) { ++j; break; }
       }
       tc_fence_after();
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);
@@ -352,6 +354,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_bf16_kernel(const Param
       if (lane == 0) mbar_arrive(bar(BAR_PFULL + t));
     }
 
+    if (!ok) pair_keep_company(pair_bar, 2 * (T - j));
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar(BAR_ODONE + t), (uint32_t)((T - 1) & 1), own_limit_only, p.status, 33, kWaitLimitCycles, abort_flag));
     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
     sMax[h * 128 + row] = l_run;

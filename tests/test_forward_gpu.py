@@ -271,3 +271,30 @@ def test_registered_workspace_entry_point(uos, pnq):
         assert ei.value.code == -4
     finally:
         mx.set_workspace(None)
+
+
+@pytest.mark.parametrize("B,H,nq,nkv", [(1, 3, 300, 1000), (4, 60, 520, 700)])
+def test_cycle_profile_build_gives_the_same_output_and_fills_its_counters(B, H, nq, nkv):
+    """The kernel compiled with cycle counters (a performance-analysis aid) computes exactly what the timed kernel
+    computes; its counters account for every tile.  Second case: the item-walking variant."""
+    import paper_2607_24377_b200 as mx
+    cfg = si.custom_config("prof", B, H, nq, nkv, 81)
+    q, k, v = si.make_all(cfg)
+    dq, dk, dv = util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v)
+    flags = mx.FLAG_UOS | mx.FLAG_PNQ
+    ws = torch.empty(mx.forward_workspace_bytes(B, H, nq, nkv, 128), dtype=torch.uint8, device="cuda")
+    want = torch.empty((B, H, nq, 128), dtype=torch.bfloat16, device="cuda")
+    mx.forward_ws(dq, dk, dv, want, B, H, nq, nkv, 128, cfg.softmax_scale, flags, ws)
+    g_out = util.guarded((B, H, nq, 128), torch.bfloat16, float("nan"))
+    g_prof = util.guarded((mx.forward_cycle_profile_bytes(B, H, nq, nkv, 128) // 8,), torch.int64, 0)
+    mx.forward_cycle_profile(dq, dk, dv, g_out.t, B, H, nq, nkv, 128, cfg.softmax_scale, flags, ws, g_prof.t)
+    assert mx.device_status(ws) == 0
+    g_out.check(); g_prof.check()
+    assert torch.equal(g_out.t, want)
+    p = g_prof.t.view(-1, 18, 16).cpu().numpy()
+    ran = p[p[:, 17, 9] > 0]
+    items = B * H * -(-(-(-nq // 128)) // 2)
+    tiles = -(-nkv // 128)
+    assert ran[:, 17, 9].sum() == items * tiles                        # the issuer saw every tile of every item
+    assert (ran[:, :16, 9].sum(axis=0) == items * tiles).all()         # and so did each of the 16 softmax warps
+    assert (ran[:, :16, 6] > 0).all() and (ran[:, 17, 8] > 0).all()
