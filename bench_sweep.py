@@ -81,6 +81,9 @@ def cycle_profile(mx, torch, cfg, dev):
            "producer_cycles_per_tile": {"loop_total": float((p[:, 16, 8:9] / tiles).mean()), "wait_free_stage": float((p[:, 16, 3:4] / tiles).mean()),
                                         "wait_free_q_buffer": float((p[:, 16, 5:6] / tiles).mean())}}
     rep["softmax_cycles_per_tile"]["sum"] = float(per_tile.sum(axis=2).mean())
+    for g in (0, 1):            # the two softmax groups (query tile 0: warps 0-7, query tile 1: warps 8-15) separately
+        pg = per_tile[:, 8 * g:8 * g + 8, :]
+        rep[f"softmax_group{g}_cycles_per_tile"] = {SOFTMAX_PHASES[i]: float(pg[:, :, i].mean()) for i in range(8)}
     rep["issuer_cycles_per_tile"]["issuing"] = rep["issuer_cycles_per_tile"]["loop_total"] - sum(
         v for k_, v in rep["issuer_cycles_per_tile"].items() if k_.startswith("wait"))
     return rep

@@ -309,14 +309,29 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
         tc_cp_sf(tmem + kColSFV + 4, sbase + kOffSFOnes);        // scales of the ones rows, both slots
         tc_cp_sf(tmem + kColSFV + 12, sbase + kOffSFOnes);
       }
+      // K-hat of tile f has landed: its scale atom goes to tensor memory (slot f & 1 was last read by the score products
+      // of tile f - 2, issued before).  Kept apart from the wait for the score buffer, so that nothing but that wait
+      // stands between "the other group has taken its scores" and the next score product.
+      auto k_ready = [&](int f) {
+        const int s = f % kStages;
+        if (!MBAR_WAIT_ROLE(bar(BAR_KFULL + s), (uint32_t)((f / kStages) & 1), abort_flag, p.status, 22)) return false;
+        tc_fence_after();
+        tc_cp_sf(tmem + kColSFK + 4 * (f & 1), sbase + kOffSFK + s * kTileScaleBytes);
+        return true;
+      };
+      // V-hat's scale atom of tile f (its stage has landed together with K-hat's; slot f & 1 was last read by the output
+      // products of tile f - 2)
+      auto v_scales = [&](int f) { tc_cp_sf(tmem + kColSFV + 8 * (f & 1), sbase + kOffSFV + (f % kStages) * kTileScaleBytes); };
       if (!kPersist) {
         // prologue: S(0,0), S(1,0), S(0,1)
-        ok = ok && wait_kv(0, true);
-        if (ok) gemm1(0, 0, 0, 0);
+        ok = ok && k_ready(0);
+        if (ok) { v_scales(0); gemm1(0, 0, 0, 0); }
         ok = ok && wait_sfree();
         if (ok) gemm1(1, 0, 0, 0);
         if (T > 1) {
-          ok = ok && wait_kv(1, false);
+          ok = ok && k_ready(1);
+          if (ok) v_scales(1);
+          ok = ok && wait_sfree();
           if (ok) gemm1(0, 0, 1, 1);
         }
         // unrolled by the number of stages: stage indices, parities and descriptor offsets become constants, and the
@@ -333,16 +348,21 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
             if (!ok) break;
             gemm1(1, 0, j + 1, j + 1);
           }
+          if (j + 2 < T) {                           // off the critical chain: the thread would wait for P-hat here anyway
+            ok = k_ready(j + 2);
+            if (!ok) break;
+          }
           ok = MBAR_WAIT_ROLE(bar(BAR_PFULL + 1), (uint32_t)(j & 1), abort_flag, p.status, 26);
           if (!ok) break;
           tc_fence_after();
           gemm2(1, 0, j, j);
-          tc_commit(bar(BAR_KEMPTY + s));            // the last reader of stage s: K_j and V_j may be overwritten
           if (j + 2 < T) {
-            ok = wait_kv(j + 2, false);
+            ok = wait_sfree();
             if (!ok) break;
             gemm1(0, 0, j + 2, j + 2);
           }
+          tc_commit(bar(BAR_KEMPTY + s));            // K_j and V_j may be overwritten once everything issued so far has completed
+          if (j + 2 < T) v_scales(j + 2);
         }
       } else {
         // The same instruction stream over all tiles of all items of this CTA, f = 0 .. F_end - 1: the scores of
