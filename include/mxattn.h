@@ -41,11 +41,11 @@ typedef enum { MXATTN_MODE_OCP = 0, MXATTN_MODE_UOS = 1 } mxattn_mode;
 /* OR-able into `mode` of the quantizer: first apply the fixed orthogonal Hadamard rotation
  * y = x H_128 / sqrt(128) to every row (paper Algorithm 2, lines 1-2; Section 4.3), then quantize y.
  * H_128 is the Sylvester matrix, H[i][j] = (-1)^popcount(i & j).  There is no rounding to bf16 between the rotation
- * and the quantizer.  Evaluation order of this library (not part of the paper's definition): fp32 throughout, the
- * fast Walsh-Hadamard butterfly with strides 1, 2, ..., 64, each stage (a, b) -> (a + b, a - b), then one multiply by
- * fl32(1/sqrt(128)).  Against the exact product rounded once to fp32 this carries about 1e-7 of relative rounding
- * noise, which can move a code or a scale byte only where a rotated value sits that close to a rounding boundary
- * (none in 1.6e7 values of the test recipes).
+ * and the quantizer.  How this library evaluates it (not part of the paper's definition): x H_128 as a bf16 matrix
+ * product on the tensor core -- the entries of H are +-1, so every product is exact and the sums are accumulated in
+ * fp32 -- followed by one fp32 multiply by fl32(1/sqrt(128)).  Against the exact product rounded once to fp32 this
+ * carries about 1e-7 of relative rounding noise, which can move a code or a scale byte only where a rotated value
+ * sits that close to a rounding boundary (none in 1.6e7 values of the test recipes; the tests bound the rate by 1e-5).
  * Only block_axis 1 with cols == 128. */
 enum { MXATTN_MODE_HADAMARD = 0x100 };
 
@@ -338,6 +338,11 @@ int mxattn_forward_static(const void* q, const void* k, const void* v, void* o,
 int mxattn_probe_fp4_gemm(const void* a_codes, const void* a_scales, const void* b_codes, const void* b_scales,
                           void* c, int64_t M, int64_t N, int64_t K, int64_t k_steps, int resident, int out_fp32,
                           int tile_n, void* status, void* stream);
+
+/* Synchronizes `stream`, then copies to *host_out (host pointer) the status word of the rotating quantizer, the one
+ * quantize kernel with a device-side wait (for its tensor-core product): 0 = no bounded wait of it ever expired in
+ * this process on the current device. */
+int mxattn_quantizer_status(int* host_out, void* stream);
 
 /* Synchronizes `stream`, then copies the workspace's status word to *host_out (host pointer):
  * 0 = no bounded wait expired since the workspace was last used by a forward. */

@@ -176,24 +176,3 @@ def hadamard_rotate(x: np.ndarray) -> np.ndarray:
     x64 = np.asarray(x, dtype=np.float64)
     n = x64.shape[-1]
     return ((x64 @ hadamard_matrix(n)) / np.sqrt(np.float64(n))).astype(np.float32)
-
-
-def hadamard_rotate_fwht_f32(x: np.ndarray) -> np.ndarray:
-    """SECONDARY check, not the definition: the same rotation evaluated entirely in fp32 in the order the
-    library documents for its kernel -- fast Walsh-Hadamard butterfly with strides 1, 2, 4, ..., n/2, each
-    stage (a, b) -> (a + b, a - b) in IEEE fp32, then one fp32 multiply by fl32(1/sqrt(n)).  It differs from
-    `hadamard_rotate` by fp32 rounding noise (about 1e-7 relative), which moves a quantized code only when a
-    value sits that close to a rounding boundary.  Tests use it to check that the kernel follows its documented
-    evaluation order; parity with the paper's definition is judged against `hadamard_rotate`."""
-    y = np.array(x, dtype=np.float32, copy=True)
-    n = y.shape[-1]
-    assert n & (n - 1) == 0
-    stride = 1
-    while stride < n:
-        v = y.reshape(y.shape[:-1] + (n // (2 * stride), 2, stride))
-        a = v[..., 0, :].copy()
-        b = v[..., 1, :].copy()
-        v[..., 0, :] = a + b
-        v[..., 1, :] = a - b
-        stride *= 2
-    return y * np.float32(1.0 / np.sqrt(np.float64(n)))

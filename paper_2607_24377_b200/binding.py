@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.mxattn_forward_host_arena_bytes.restype = sz
         L.mxattn_forward_host.argtypes = [vp, vp, vp, vp, ci, ci, i64, i64, ci, cf, cu, vp, sz, vp]
         L.mxattn_probe_fp4_gemm.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, ci, ci, ci, vp, vp]
+        L.mxattn_quantizer_status.argtypes = [ctypes.POINTER(ctypes.c_int), vp]
         L.mxattn_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), vp]
         L.mxattn_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.mxattn_selftest_pair_abandon.argtypes = [vp, i64, ci, vp]
@@ -225,6 +226,12 @@ def probe_fp4_gemm(a_codes, a_scales, b_codes, b_scales, c, M, N, K, k_steps, re
     _check(lib().mxattn_probe_fp4_gemm(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), _ptr(c), M, N, K,
                                        k_steps, int(resident), int(out_fp32), int(tile_n), _ptr(status), _stream()),
            "mxattn_probe_fp4_gemm")
+
+
+def quantizer_status() -> int:
+    out = ctypes.c_int(0)
+    _check(lib().mxattn_quantizer_status(ctypes.byref(out), _stream()), "mxattn_quantizer_status")
+    return out.value
 
 
 def device_status(workspace) -> int:

@@ -1,15 +1,18 @@
 // MXFP4 block quantization kernels (paper Section 2, Eq. 4-7; Algorithm 1) for sm_100a.
 //
-// Both kernels are HBM-bound streaming passes: 2 bytes read, 0.5 + 1/32 bytes written per element.
+// All kernels are HBM-bound streaming passes: 2 bytes read, 0.5 + 1/32 bytes written per element.
 //   axis 1 (Q, K): a block is 32 consecutive bf16 of one row.  One thread owns 8 elements (one
 //     128-bit load); the 4 threads of a block combine their maxima with two shuffles.
 //   axis 0 (V): a block is 32 consecutive rows (tokens) of one column.  A CTA stages a
 //     128-token x 128-column slab in shared memory with coalesced 128-bit loads, quantizes down
 //     the columns, and writes the transposed codes through a shared-memory staging tile so that
 //     the global stores stay 128-bit.
+//   axis 1 with the Hadamard rotation of Algorithm 2 (Q, K): the rotation of a 128-row tile is one bf16 matrix
+//     product with the +-1 matrix on the tensor core; the quantizer reads the rotated rows out of tensor memory.
 #include <string.h>
 
 #include "common.cuh"
+#include "tc_helpers.cuh"
 
 namespace mxattn {
 
@@ -26,37 +29,6 @@ __device__ __forceinline__ uint32_t absmax_bf16x8(const uint4& v) {
 __device__ __forceinline__ uint32_t quantize_bf16x8(const uint4& v, float inv) {
   return pack_e2m1x8(bf16lo(v.x) * inv, bf16hi(v.x) * inv, bf16lo(v.y) * inv, bf16hi(v.y) * inv,
                      bf16lo(v.z) * inv, bf16hi(v.z) * inv, bf16lo(v.w) * inv, bf16hi(v.w) * inv);
-}
-
-// Packed fp32x2 arithmetic (two IEEE round-to-nearest fp32 operations per instruction; each half gives
-// exactly the result of the scalar instruction).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
 }
 
 // One 16-byte chunk (8 bf16) -> packed codes and the block's shared exponent; the four lanes of a
@@ -152,118 +124,180 @@ quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ c
 }
 
 // ------------------------------------------------------------------------------------------
-// Axis 1 with the Hadamard rotation (cols == 128), both layouts.  A CTA takes 128 consecutive rows;
-// FOUR lanes share a row and each holds 32 of its elements: lane q (0..3) loads the 16-byte chunks
-// q, q + 4, q + 8, q + 12, so element index = 32 u + 8 q + i with u = 0..3 the chunk number within the
-// lane and i = 0..7.  The butterfly stages of strides 1, 2, 4 (bits of i) and 32, 64 (bits of u) stay
-// inside the thread; only strides 8 and 16 (bits of q) cross lanes -- two shuffle stages per row
-// instead of the four that an 8-elements-per-lane split needs.  Stage order (ascending strides) and
-// the fp32 arithmetic (every stage (a, b) -> (a + b, a - b) with a the lower index, then one multiply by
-// fl32(1/sqrt(128))) are part of the definition, because the result feeds a rounding decision.  The MX block
-// u is the chunk u of the four lanes: its maximum takes two more shuffles, its codes are one word per
-// lane, its scale byte is written (with the row's other three) by lane 0.
-// kRuleKind: 0 = OCP floor rule, 1 = UOS (boundary 7.25, the mantissa compare of shared_exponent), 2 = the
-// boundary passed in `rule` (this kernel is bound by instruction issue, so the common rules are compiled in).
+// Axis 1 with the Hadamard rotation on the tensor core (cols == 128), both layouts.  The rotation of a 128-row tile,
+// Y = X H_128, is one 128 x 128 x 128 bf16 matrix product: X is bf16 as given, the entries of H are +-1 (exact in
+// bf16), every product is exact and the sums are accumulated in fp32 by tcgen05.mma kind::f16 into tensor memory.
+// Two threads then share a row of Y (64 columns = two blocks each): scale by fl32(1/sqrt(128)), block maxima, quantize.
+// Against the exact product rounded once to fp32 the tensor core's fp32 accumulation carries rounding noise of about
+// 1e-7 relative, which moves a code only where a value sits that close to a rounding boundary.
+//
+// Persistent CTAs (two per SM, 256 threads) walk the tiles.  H (32 KiB, generated once per CTA) and two X buffers
+// (32 KiB each) sit in shared memory as K-major operand tiles (two 64-element K halves, 128-byte swizzle); X arrives
+// by 16-byte asynchronous copies straight into its swizzled place; two accumulators of 128 tensor-memory columns
+// alternate, so that the product of tile i runs while tile i - 1 is quantized and tile i + 1 is fetched.
+namespace rot {
+using namespace fwd;
+constexpr int kThreads = 256;
+constexpr int kHalf = 16384;                              // one K half of an operand tile: 128 rows x 128 bytes
+constexpr int kOffH = 4 * kHalf;                          // after the two X buffers
+constexpr int kOffBar = 6 * kHalf;
+constexpr int kSmemBytes = kOffBar + 64 + 1024;           // + barriers, slots, slack for the 1024-byte alignment
+__device__ int g_status = 0;                               // non-zero if a bounded wait for a product ever ran out
+
+__device__ __forceinline__ int half_chunk_offset(int r, int c) { return r * 128 + ((c ^ (r & 7)) << 4); }
+
 template <bool kTileLayout, int kRuleKind>
-__global__ void __launch_bounds__(kQThreads)
-quantize_axis1_rot_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
-                          uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
-  const int tid = threadIdx.x;
-  const int q = tid & 3, rr = tid >> 2;              // lane within the row's quad; row within a 64-row pass
-  // tile layout: grid = (row tiles, batch), `rows` per batch entry; canonical: grid = row groups, `rows` in total
-  const int64_t row0 = (int64_t)blockIdx.x * kTile;
-  const uint4* src = in + ((kTileLayout ? (int64_t)blockIdx.y * rows : 0) + row0) * 16;     // 16 chunks per row
-  const int rows_here = (int)min((int64_t)kTile, rows - row0);
-  uint4 v[2][4];
+__global__ void __launch_bounds__(kThreads, 2)
+quantize_axis1_rot_tc_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                             int64_t rows, int tiles_per_matrix, int n_tiles, uint32_t rule) {
+  // tile layout: `rows` per matrix of the batch, tile = matrix * tiles_per_matrix + tile within the matrix;
+  // canonical: one matrix of `rows` rows (the batch is contiguous), tiles_per_matrix == n_tiles
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + kOffBar;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffBar + 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffBar + 24);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int n_my = ((int)blockIdx.x < n_tiles) ? (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+  auto tile_rows = [&](int tile, int64_t* first_row) {       // rows of the input this tile covers
+    const int m = tile / tiles_per_matrix, t = tile - m * tiles_per_matrix;
+    *first_row = (int64_t)m * rows + (int64_t)t * kTile;
+    return (int)min((int64_t)kTile, rows - (int64_t)t * kTile);
+  };
+  auto fetch = [&](int tile, int buf) {                       // X tile -> shared memory, zero beyond the matrix
+    int64_t first;
+    const int here = tile_rows(tile, &first);
+    const uint4* src = in + first * 16;
 #pragma unroll
-  for (int k = 0; k < 2; ++k)
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int r = k * 64 + rr;
-      v[k][u] = r < rows_here ? __ldg(src + r * 16 + 4 * u + q) : make_uint4(0u, 0u, 0u, 0u);
+    for (int k = 0; k < 8; ++k) {
+      const int chunk = k * kThreads + tid;
+      const int r = chunk >> 4, cc = chunk & 15;
+      const uint32_t dst = sbase + buf * 2 * kHalf + (cc >> 3) * kHalf + half_chunk_offset(r, cc & 7);
+      const bool valid = r < here;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(valid ? src + chunk : in), "r"(valid ? 16 : 0) : "memory");
     }
-  const int64_t tile = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
-  const uint64_t sgn1 = (q & 1) ? pack2(-1.0f, -1.0f) : pack2(1.0f, 1.0f);
-  const uint64_t sgn2 = (q & 2) ? pack2(-1.0f, -1.0f) : pack2(1.0f, 1.0f);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  if (tid == 0) {
+    mbar_init(bar0, 1); mbar_init(bar0 + 8, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (n_my > 0) fetch(blockIdx.x, 0);
+  // H as the B operand: B[n][k] = H[k][n] = (-1)^popcount(n & k); chunk (n, cc) holds k = 8 cc .. 8 cc + 7
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    const int r = k * 64 + rr;
-    // the 32 values as 16 packed pairs: pair j = elements (2j, 2j + 1) of the thread
-    uint64_t pr[16];
+  for (int k = 0; k < 8; ++k) {
+    const int chunk = k * kThreads + tid;
+    const int n = chunk >> 4, cc = chunk & 15;
+    const uint32_t base_par = (uint32_t)__popc(n & (cc << 3)) & 1u;
+    uint32_t w[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint4& w = v[k][u];
-      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        // stride 1 on the way in: (a, b) -> (a + b, a - b)
-        const float a = bf16lo(ww[j]), b = bf16hi(ww[j]);
-        pr[4 * u + j] = pack2(__fadd_rn(a, b), __fsub_rn(a, b));
-      }
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t p0 = (base_par ^ ((uint32_t)__popc(n & (2 * i)) & 1u)), p1 = (base_par ^ ((uint32_t)__popc(n & (2 * i + 1)) & 1u));
+      w[i] = (0x3F80u | (p0 << 15)) | ((0x3F80u | (p1 << 15)) << 16);       // bf16 +1 / -1
     }
-    // strides 2, 4 (pair strides 1, 2): inside each chunk, two elements per instruction
+    *reinterpret_cast<uint4*>(smem + kOffH + (cc >> 3) * kHalf + half_chunk_offset(n, cc & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  // epilogue of one tile: this thread's half row (row r, columns 64 h .. 64 h + 63) out of accumulator `buf`
+  const int r = (warp & 3) * 32 + (tid & 31), h = warp >> 2;
+  auto quantize_tile = [&](int tile, int buf) {
+    int64_t first;
+    const int here = tile_rows(tile, &first);
+    const uint32_t t_row = tmem + 128 * buf + ((uint32_t)((warp & 3) * 32) << 16) + 64 * h;
+    uint32_t sf = 0;
 #pragma unroll
-    for (int st = 1; st < 4; st <<= 1)
+    for (int u = 0; u < 2; ++u) {
+      uint32_t acc[32];
+      TMEM_LD32(t_row + 32 * u, acc);
+      tmem_ld_wait();
+      float y[32], mf = 0.0f;
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if ((j & st) == 0) {
-          const uint64_t a = pr[j], b = pr[j + st];
-          pr[j] = add2(a, b);
-          pr[j + st] = sub2(a, b);
-        }
-    // strides 8, 16: across the quad.  The lower lane gets a + b = own * 1 + other, the upper one
-    // a - b = own * (-1) + other (the product is exact, so the fma rounds like the add / subtract).
-#pragma unroll
-    for (int j = 0; j < 16; ++j) pr[j] = fma2(pr[j], sgn1, __shfl_xor_sync(0xFFFFFFFFu, pr[j], 1));
-#pragma unroll
-    for (int j = 0; j < 16; ++j) pr[j] = fma2(pr[j], sgn2, __shfl_xor_sync(0xFFFFFFFFu, pr[j], 2));
-    // strides 32, 64 (pair strides 4, 8): across the thread's chunks
-#pragma unroll
-    for (int st = 4; st < 16; st <<= 1)
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if ((j & st) == 0) {
-          const uint64_t a = pr[j], b = pr[j + st];
-          pr[j] = add2(a, b);
-          pr[j + st] = sub2(a, b);
-        }
-    uint32_t word[4], sf = 0;
-    const uint64_t norm2 = pack2(0.08838834764831845f, 0.08838834764831845f);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      float mf = 0.0f;                               // max |.| as a float: the operand modifiers make |x| free
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        pr[4 * u + j] = mul2(pr[4 * u + j], norm2);
-        float lo, hi;
-        unpack2(pr[4 * u + j], lo, hi);
-        mf = fmaxf(fmaxf(mf, fabsf(lo)), fabsf(hi));
+      for (int i = 0; i < 32; ++i) {
+        y[i] = __fmul_rn(__uint_as_float(acc[i]), 0.08838834764831845f);
+        mf = fmaxf(mf, fabsf(y[i]));
       }
-      mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 1));
-      mf = fmaxf(mf, __shfl_xor_sync(0xFFFFFFFFu, mf, 2));
-      const int e = kRuleKind == 2 ? shared_exponent_ceil(__float_as_uint(mf), rule)
-                                   : shared_exponent(__float_as_uint(mf), kRuleKind == 1);
+      const int e = kRuleKind == 2 ? shared_exponent_ceil(__float_as_uint(mf), rule) : shared_exponent(__float_as_uint(mf), kRuleKind == 1);
       const float inv = pow2_neg(e);
-      const uint64_t inv2 = pack2(inv, inv);
-      float x[8];
+      uint32_t wd[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) unpack2(mul2(pr[4 * u + j], inv2), x[2 * j], x[2 * j + 1]);
-      word[u] = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
+      for (int g = 0; g < 4; ++g)
+        wd[g] = pack_e2m1x8(y[8 * g] * inv, y[8 * g + 1] * inv, y[8 * g + 2] * inv, y[8 * g + 3] * inv,
+                            y[8 * g + 4] * inv, y[8 * g + 5] * inv, y[8 * g + 6] * inv, y[8 * g + 7] * inv);
       sf |= (uint32_t)(e + 127) << (8 * u);
+      const int blk = 2 * h + u;
+      if (kTileLayout)
+        *reinterpret_cast<uint4*>(codes + (int64_t)tile * kTileCodeBytes + tile_code_offset(r, blk)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+      else if (r < here)
+        *reinterpret_cast<uint4*>(codes + (first + r) * 64 + 16 * blk) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
     }
-    if (kTileLayout) {
-      uint32_t* ctile = reinterpret_cast<uint32_t*>(codes + tile * kTileCodeBytes);
+    if (kTileLayout)
+      *reinterpret_cast<uint16_t*>(scales + (int64_t)tile * kTileScaleBytes + tile_scale_offset(r, 2 * h)) = (uint16_t)sf;
+    else if (r < here)
+      *reinterpret_cast<uint16_t*>(scales + (first + r) * 4 + 2 * h) = (uint16_t)sf;
+  };
+
+  bool ok = true;
+  for (int i = 0; i < n_my && ok; ++i) {
+    const int tile = (int)blockIdx.x + i * (int)gridDim.x;
+    if (i > 0) {                                       // the product of tile i - 1 is complete: its X buffer is free, its accumulator full
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar0 + 8 * ((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, &g_status, 51));
+      if (!ok) break;
+      tc_fence_after();
+    }
+    if (i + 1 < n_my) {                                // fetch tile i + 1 as early as its buffer allows
+      fetch(tile + (int)gridDim.x, (i + 1) & 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");        // X(i) has landed; X(i + 1) stays in flight
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();                                               // X(i) is there for every thread; accumulator i & 1 has been read out
+    tc_fence_after();
+    if (tid == 0) {
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);     // 8-row groups 1024 B apart, 128-byte swizzle
+      constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);   // fp32 accumulate, bf16 x bf16, N = 128, M = 128
+      const uint32_t a = (sbase + (i & 1) * 2 * kHalf) >> 4, b = (sbase + kOffH) >> 4;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) ctile[tile_code_offset(r, u) / 4 + q] = word[u];
-      if (q == 0) *reinterpret_cast<uint32_t*>(scales + tile * kTileScaleBytes + tile_scale_offset(r, 0)) = sf;
-    } else if (r < rows_here) {
-      uint32_t* crow = reinterpret_cast<uint32_t*>(codes) + (row0 + r) * 16;
-#pragma unroll
-      for (int u = 0; u < 4; ++u) crow[4 * u + q] = word[u];
-      if (q == 0) *reinterpret_cast<uint32_t*>(scales + (row0 + r) * 4) = sf;
+      for (int k = 0; k < 8; ++k) {                    // K = 16 per instruction: 4 steps of 32 bytes per 64-element half
+        const uint32_t off = (uint32_t)(k >> 2) * (kHalf >> 4) + (uint32_t)(k & 3) * 2;
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(tmem + 128 * (i & 1)), "l"(((uint64_t)kDescHi << 32) | (a + off)), "l"(((uint64_t)kDescHi << 32) | (b + off)),
+                       "r"(kIdesc), "r"(k > 0 ? 1u : 0u) : "memory");
+      }
+      tc_commit(bar0 + 8 * (i & 1));
+    }
+    if (i > 0) quantize_tile(tile - (int)gridDim.x, (i - 1) & 1);
+  }
+  if (ok && n_my > 0) {
+    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar0 + 8 * ((n_my - 1) & 1), (uint32_t)(((n_my - 1) >> 1) & 1), abort_flag, &g_status, 51));
+    if (ok) {
+      tc_fence_after();
+      quantize_tile((int)blockIdx.x + (n_my - 1) * (int)gridDim.x, (n_my - 1) & 1);
     }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+  }
 }
+}  // namespace rot
 
 // ------------------------------------------------------------------------------------------
 // Axis 0.  256 threads; a CTA stages a 32 KiB slab of the input in shared memory:
@@ -373,6 +407,17 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
 }
 
 // ------------------------------------------------------------------------------------------
+// persistent grid of the rotating quantizer: two CTAs per SM
+static int rot_grid() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n = 2 * v;
+  }
+  return n;
+}
+
 int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, int64_t rows,
                     int64_t cols, int block_axis, int mode, int layout, cudaStream_t stream,
                     uint32_t rule_override) {
@@ -400,9 +445,13 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
       if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
       dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
       if (rotate) {
-        auto kern = rule == kRuleOcp ? quantize_axis1_rot_kernel<true, 0>
-                  : rule == kRuleUos ? quantize_axis1_rot_kernel<true, 1> : quantize_axis1_rot_kernel<true, 2>;
-        kern<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, rows, rule);
+        auto kern = rule == kRuleOcp ? rot::quantize_axis1_rot_tc_kernel<true, 0>
+                  : rule == kRuleUos ? rot::quantize_axis1_rot_tc_kernel<true, 1> : rot::quantize_axis1_rot_tc_kernel<true, 2>;
+        const int64_t n_tiles = batch * (rows_pad / kTile);
+        if (n_tiles > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, rot::kSmemBytes) != cudaSuccess) return MXATTN_ECUDA;
+        kern<<<(unsigned)min((int64_t)rot_grid(), n_tiles), rot::kThreads, rot::kSmemBytes, stream>>>(
+            (const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, rows, (int)(rows_pad / kTile), (int)n_tiles, rule);
       } else
         quantize_axis1_tile_kernel<<<grid, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes,
                                                                           (uint8_t*)scales, rows, rule);
@@ -410,10 +459,11 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
       if (rotate) {                                  // cols == 128 here: batch * rows rows of 16 chunks
         const int64_t groups = (batch * rows + kTile - 1) / kTile;
         if (groups > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
-        auto kern = rule == kRuleOcp ? quantize_axis1_rot_kernel<false, 0>
-                  : rule == kRuleUos ? quantize_axis1_rot_kernel<false, 1> : quantize_axis1_rot_kernel<false, 2>;
-        kern<<<(unsigned)groups, kQThreads, 0, stream>>>((const uint4*)in, (uint8_t*)codes, (uint8_t*)scales,
-                                                         batch * rows, rule);
+        auto kern = rule == kRuleOcp ? rot::quantize_axis1_rot_tc_kernel<false, 0>
+                  : rule == kRuleUos ? rot::quantize_axis1_rot_tc_kernel<false, 1> : rot::quantize_axis1_rot_tc_kernel<false, 2>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, rot::kSmemBytes) != cudaSuccess) return MXATTN_ECUDA;
+        kern<<<(unsigned)min((int64_t)rot_grid(), groups), rot::kThreads, rot::kSmemBytes, stream>>>(
+            (const uint4*)in, (uint8_t*)codes, (uint8_t*)scales, batch * rows, (int)groups, (int)groups, rule);
       } else
         quantize_axis1_kernel<<<(unsigned)blocks, kQThreads, 0, stream>>>(
             (const uint4*)in, (uint32_t*)codes, (uint8_t*)scales, n_chunks, rule);
@@ -457,4 +507,11 @@ extern "C" int mxattn_quantize_mxfp4_qmax(const void* in, void* codes, void* e8m
   memcpy(&bits, &qmax, sizeof bits);
   return mxattn::launch_quantize(in, codes, e8m0_scales, batch, rows, cols, block_axis, MXATTN_MODE_UOS, layout,
                                  (cudaStream_t)stream, bits);
+}
+
+extern "C" int mxattn_quantizer_status(int* host_out, void* stream) {
+  if (!host_out) return MXATTN_EINVAL;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MXATTN_ECUDA;
+  if (cudaMemcpyFromSymbol(host_out, mxattn::rot::g_status, sizeof(int)) != cudaSuccess) return MXATTN_ECUDA;
+  return MXATTN_OK;
 }

@@ -182,21 +182,26 @@ def test_hadamard_rotated_quantization_against_the_plain_definition(recipe, rows
 
 
 @pytest.mark.parametrize("mode", [0, 1])
-@pytest.mark.parametrize("rows", [1, 100, 1024, 4099])
-def test_hadamard_rotated_quantization_follows_its_documented_evaluation_order(rows, mode):
-    # secondary check: the kernel's fp32 evaluation order (include/mxattn.h, MXATTN_MODE_HADAMARD) is reproduced bit for bit;
-    # parity with the paper's definition is the test above
-    bits = gaussian_bits(rows, 128, 300 + rows + mode)
-    bits[::5, 7] = si.f32_to_bf16_bits(np.full(len(bits[::5]), 37.5, np.float32))      # a channel outlier
-    x = si.bf16_bits_to_f32(bits)
-    want_c, want_s = mxfp4.quantize_matrix_canonical(mxfp4.hadamard_rotate_fwht_f32(x).astype(np.float64), 1, RULE[mode])
-    got_c, got_s = _rotated_gpu(bits, rows, mode)
-    assert np.array_equal(got_s, want_s)
-    assert np.array_equal(got_c, want_c)
-    # tile layout: same values, permuted
-    tc, ts = _rotated_gpu(bits, rows, mode, layout_tile=True)
-    wc, ws = util.canonical_to_tile_axis1(want_c, want_s)
-    assert np.array_equal(ts[0], ws) and np.array_equal(tc[0], wc)
+@pytest.mark.parametrize("batch,rows", [(1, 1), (3, 100), (2, 1024), (1, 4099), (5, 300)])
+def test_hadamard_rotated_quantization_tile_layout_is_a_permutation_of_the_canonical_one(batch, rows, mode):
+    import paper_2607_24377_b200 as mx
+    bits = np.stack([gaussian_bits(rows, 128, 300 + rows + mode + b) for b in range(batch)])
+    bits[:, ::5, 7] = si.f32_to_bf16_bits(np.full(bits[:, ::5, 7].shape, 37.5, np.float32))      # a channel outlier
+    nt = -(-rows // 128)
+    gc = util.guarded((batch, rows, 64), torch.uint8, 0xAA); gs = util.guarded((batch, rows, 4), torch.uint8, 0xAA)
+    mx.quantize_mxfp4_batched(util.to_dev_bf16(bits), gc.t, gs.t, batch, rows, 128, 1, mode | mx.MODE_HADAMARD, mx.LAYOUT_CANONICAL)
+    tc = util.guarded((batch, nt, 8192), torch.uint8, 0xAA); ts = util.guarded((batch, nt, 512), torch.uint8, 0xAA)
+    mx.quantize_mxfp4_batched(util.to_dev_bf16(bits), tc.t, ts.t, batch, rows, 128, 1, mode | mx.MODE_HADAMARD, mx.LAYOUT_TILE)
+    for g in (gc, gs, tc, ts):
+        g.check()
+    assert mx.quantizer_status() == 0
+    for b in range(batch):
+        wc, ws = util.canonical_to_tile_axis1(gc.t[b].cpu().numpy(), gs.t[b].cpu().numpy())
+        assert np.array_equal(ts.t[b].cpu().numpy(), ws) and np.array_equal(tc.t[b].cpu().numpy(), wc)
+        # and the canonical output is the plain-definition oracle's (these sizes are far too small for a boundary case)
+        x = si.bf16_bits_to_f32(bits[b])
+        want_c, want_s = mxfp4.quantize_matrix_canonical(mxfp4.hadamard_rotate(x).astype(np.float64), 1, RULE[mode])
+        assert np.array_equal(gs.t[b].cpu().numpy(), want_s) and np.array_equal(gc.t[b].cpu().numpy(), want_c)
 
 
 def test_rotation_is_refused_where_it_is_not_defined():
