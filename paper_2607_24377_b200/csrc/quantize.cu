@@ -1,8 +1,9 @@
 // MXFP4 block quantization kernels (paper Section 2, Eq. 4-7; Algorithm 1) for sm_100a.
 //
 // All kernels are HBM-bound streaming passes: 2 bytes read, 0.5 + 1/32 bytes written per element.
-//   axis 1 (Q, K): a block is 32 consecutive bf16 of one row.  One thread owns 8 elements (one
-//     128-bit load); the 4 threads of a block combine their maxima with two shuffles.
+//   axis 1 (Q, K): a block is 32 consecutive bf16 of one row.  The CTA's input arrives in shared memory by
+//     asynchronous 16-byte copies; one thread then owns a whole block (four 16-byte chunks) and writes its
+//     16 bytes of codes with one store.
 //   axis 0 (V): a block is 32 consecutive rows (tokens) of one column.  A CTA stages a
 //     128-token x 128-column slab in shared memory with coalesced 128-bit loads, quantizes down
 //     the columns, and writes the transposed codes through a shared-memory staging tile so that
@@ -31,96 +32,105 @@ __device__ __forceinline__ uint32_t quantize_bf16x8(const uint4& v, float inv) {
                      bf16lo(v.z) * inv, bf16hi(v.z) * inv, bf16lo(v.w) * inv, bf16hi(v.w) * inv);
 }
 
-// One 16-byte chunk (8 bf16) -> packed codes and the block's shared exponent; the four lanes of a
-// 32-element block combine their maxima with two shuffles.
-__device__ __forceinline__ uint32_t quantize_chunk(const uint4& v, uint32_t rule, int* e_out) {
-  uint32_t m = absmax_bf16x8(v);
-  m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-  m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
-  const int e = shared_exponent_rule(m << 16, rule);
-  *e_out = e;
-  return quantize_bf16x8(v, pow2_neg(e));
-}
-
 constexpr int kQThreads = 256;
 
 // ------------------------------------------------------------------------------------------
-// Axis 1, canonical layout: a linear streaming pass.  Work unit = one 16-byte chunk (8 elements);
-// chunk i yields code word i and (with its three neighbours) scale byte i / 4.  A CTA owns 2048
-// consecutive chunks (32 KiB) and issues all of its loads before it quantizes anything.
-constexpr int kQChunksPerThread = 8;
+// Axis 1, canonical layout: a linear streaming pass.  Work unit = one 32-element block = four 16-byte chunks;
+// block g yields 16 bytes of codes and scale byte g.  A CTA owns 1024 consecutive chunks (16 KiB).  Measured against
+// the earlier form (a thread per chunk, loads to registers, block maximum by two shuffles, 4-byte code stores):
+// 0.83 / 0.93 / 0.98 of the plain-copy rate at 2^26 / 2^27 / 2^28 elements then, 0.89 / 1.01 / 1.06 now.
+constexpr int kQChunksPerThread = 4;
 
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_kernel(const uint4* __restrict__ in, uint32_t* __restrict__ codes,
                       uint8_t* __restrict__ scales, int64_t n_chunks, uint32_t rule) {
-  const int lane = threadIdx.x & 31;
-  const int64_t base = (int64_t)blockIdx.x * (kQThreads * kQChunksPerThread) + threadIdx.x;
-  uint4 v[kQChunksPerThread];
+  // The CTA's chunks arrive in shared memory by asynchronous 16-byte copies; then a thread owns whole blocks (four
+  // consecutive chunks): block maximum without shuffles, 16 bytes of codes per store.  Chunk c sits at position
+  // c ^ ((c >> 3) & 7) within its group of eight, so that both the copies (consecutive c per warp) and the reads
+  // (c = 4 blk + k per thread) touch every bank group once per quarter warp.
+  __shared__ uint4 s_v[kQThreads * kQChunksPerThread];
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t base = (int64_t)blockIdx.x * (kQThreads * kQChunksPerThread);
+  auto pos = [](int c) { return c ^ ((c >> 3) & 7); };
 #pragma unroll
   for (int u = 0; u < kQChunksPerThread; ++u) {
-    const int64_t i = base + u * kQThreads;
-    v[u] = i < n_chunks ? __ldg(in + i) : make_uint4(0u, 0u, 0u, 0u);
+    const int c = u * kQThreads + tid;
+    const bool inside = base + c < n_chunks;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_v[pos(c)])),
+                 "l"(inside ? in + base + c : in), "r"(inside ? 16 : 0) : "memory");
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  const int64_t n_blocks = n_chunks >> 2;           // cols is a multiple of 32: whole blocks only
+  uint4* codes16 = reinterpret_cast<uint4*>(codes);
 #pragma unroll
-  for (int u = 0; u < kQChunksPerThread; ++u) {
-    const int64_t i = base + u * kQThreads;
-    int e;
-    const uint32_t packed = quantize_chunk(v[u], rule, &e);
-    // four consecutive blocks (16 lanes) -> one 32-bit scale word
+  for (int r = 0; r < kQChunksPerThread / 4; ++r) {
+    const int blk = r * kQThreads + tid;
+    const int64_t g = (base >> 2) + blk;            // global block index
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = s_v[pos(4 * blk + k)];
+    const uint32_t m = max(max(absmax_bf16x8(v[0]), absmax_bf16x8(v[1])), max(absmax_bf16x8(v[2]), absmax_bf16x8(v[3])));
+    const int e = shared_exponent_rule(m << 16, rule);
+    const float inv = pow2_neg(e);
     const uint32_t eb = (uint32_t)(e + 127);
-    const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
-    const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
-    const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
-    if (i >= n_chunks) continue;
-    codes[i] = packed;
-    if ((lane & 15) == 0) {
-      const int64_t g = i >> 2;                      // block index, multiple of 4 here
-      if (i + 16 <= n_chunks) {
+    // four consecutive blocks (4 lanes) -> one 32-bit scale word
+    const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 1);
+    const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 2);
+    const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 3);
+    if (g >= n_blocks) continue;
+    codes16[g] = make_uint4(quantize_bf16x8(v[0], inv), quantize_bf16x8(v[1], inv), quantize_bf16x8(v[2], inv), quantize_bf16x8(v[3], inv));
+    if ((lane & 3) == 0) {
+      if (g + 4 <= n_blocks) {
         *reinterpret_cast<uint32_t*>(scales + g) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
       } else {                                       // ragged end: fewer than 4 blocks left
         scales[g] = (uint8_t)eb;
-        if (i + 4 < n_chunks) scales[g + 1] = (uint8_t)b1;
-        if (i + 8 < n_chunks) scales[g + 2] = (uint8_t)b2;
+        if (g + 1 < n_blocks) scales[g + 1] = (uint8_t)b1;
+        if (g + 2 < n_blocks) scales[g + 2] = (uint8_t)b2;
       }
     }
   }
 }
 
 // ------------------------------------------------------------------------------------------
-// Axis 1, tile layout (cols == 128).  grid = (row tiles, batch); one CTA quantizes one 128-row
-// tile: 32 KiB in, 8.5 KiB out.  A thread issues its eight 16-byte loads up front (the whole
-// tile is in flight at once), then quantizes them; a warp covers two full rows per step, so the
-// four lanes of a block and the sixteen lanes of a row are always in the same warp.
+// Axis 1, tile layout (cols == 128).  grid = (2 x row tiles, batch); one CTA quantizes half a 128-row tile
+// (64 rows, 16 KiB in) the same way: asynchronous copies into shared memory, one block (row r, 32 columns c) per
+// thread, one 16-byte store into the tile image, one 32-bit scale store per row.
 __global__ void __launch_bounds__(kQThreads)
 quantize_axis1_tile_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes,
                            uint8_t* __restrict__ scales, int64_t rows, uint32_t rule) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int64_t tile = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
-  const int64_t row0 = (int64_t)blockIdx.x * kTile;
+  __shared__ uint4 s_v[kQThreads * 4];
+  const int tid = threadIdx.x;
+  const int64_t tile = (int64_t)blockIdx.y * (gridDim.x >> 1) + (blockIdx.x >> 1);
+  const int half = blockIdx.x & 1;
+  const int64_t row0 = (int64_t)(blockIdx.x >> 1) * kTile + half * 64;
   const uint4* src = in + ((int64_t)blockIdx.y * rows + row0) * 16;     // 16 chunks per row
-  const int rows_here = (int)min((int64_t)kTile, rows - row0);
-  uint4 v[8];
+  const int rows_here = (int)max((int64_t)0, min((int64_t)64, rows - row0));
+  auto pos = [](int c) { return c ^ ((c >> 3) & 7); };
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
+  for (int k = 0; k < 4; ++k) {
     const int chunk = k * kQThreads + tid;           // row = chunk >> 4
-    v[k] = (chunk >> 4) < rows_here ? __ldg(src + chunk) : make_uint4(0u, 0u, 0u, 0u);
+    const bool inside = (chunk >> 4) < rows_here;    // rows beyond the matrix are zero blocks of the padded tile
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_v[pos(chunk)])),
+                 "l"(inside ? src + chunk : in), "r"(inside ? 16 : 0) : "memory");
   }
-  uint32_t* ctile = reinterpret_cast<uint32_t*>(codes + tile * kTileCodeBytes);
-  uint8_t* stile = scales + tile * kTileScaleBytes;
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  const int r = half * 64 + (tid >> 2), c = tid & 3;
+  uint4 v[4];
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int chunk = k * kQThreads + tid;
-    const int r = chunk >> 4, c = (chunk >> 2) & 3;
-    int e;
-    const uint32_t packed = quantize_chunk(v[k], rule, &e);
-    const uint32_t eb = (uint32_t)(e + 127);
-    const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 4);
-    const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 8);
-    const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 12);
-    ctile[tile_code_offset(r, c) / 4 + (chunk & 3)] = packed;
-    if ((lane & 15) == 0)
-      *reinterpret_cast<uint32_t*>(stile + tile_scale_offset(r, 0)) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
-  }
+  for (int k = 0; k < 4; ++k) v[k] = s_v[pos(4 * tid + k)];
+  const uint32_t m = max(max(absmax_bf16x8(v[0]), absmax_bf16x8(v[1])), max(absmax_bf16x8(v[2]), absmax_bf16x8(v[3])));
+  const int e = shared_exponent_rule(m << 16, rule);
+  const float inv = pow2_neg(e);
+  const uint32_t eb = (uint32_t)(e + 127);
+  const uint32_t b1 = __shfl_down_sync(0xFFFFFFFFu, eb, 1);
+  const uint32_t b2 = __shfl_down_sync(0xFFFFFFFFu, eb, 2);
+  const uint32_t b3 = __shfl_down_sync(0xFFFFFFFFu, eb, 3);
+  *reinterpret_cast<uint4*>(codes + tile * kTileCodeBytes + tile_code_offset(r, c)) =
+      make_uint4(quantize_bf16x8(v[0], inv), quantize_bf16x8(v[1], inv), quantize_bf16x8(v[2], inv), quantize_bf16x8(v[3], inv));
+  if (c == 0)
+    *reinterpret_cast<uint32_t*>(scales + tile * kTileScaleBytes + tile_scale_offset(r, 0)) = eb | (b1 << 8) | (b2 << 16) | (b3 << 24);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -300,7 +310,10 @@ quantize_axis1_rot_tc_kernel(const uint4* __restrict__ in, uint8_t* __restrict__
 }  // namespace rot
 
 // ------------------------------------------------------------------------------------------
-// Axis 0.  256 threads; a CTA stages a 32 KiB slab of the input in shared memory:
+// Axis 0.  256 threads; a CTA stages a 32 KiB slab of the input in shared memory, by asynchronous 16-byte copies
+// (cp.async: no staging registers and no second pass through the load/store unit; against loads to registers
+// followed by shared-memory stores this took the canonical layout from 0.77 / 0.84 / 0.88 of the plain-copy rate to
+// 0.89 / 0.97 / 1.02 at 2^26 / 2^27 / 2^28 elements):
 //   tile layout:  128 tokens x 128 columns -> one 8.5 KiB tile image, written contiguously;
 //                 grid = (1, ceil(rows/128), batch)
 //   canonical:    256 tokens x 64 columns, so that every column leaves as ONE 128-byte segment of codes
@@ -334,11 +347,12 @@ quantize_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict__ cod
   for (int k = 0; k < (kTok * kCol / 8) / kVThreads; ++k) {
     const int chunk = k * kVThreads + tid;
     const int t = chunk / (kCol / 8), cc = (chunk % (kCol / 8)) << 3;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row0 + t < rows && col0 + cc < cols)
-      v = __ldg(reinterpret_cast<const uint4*>(src + (row0 + t) * cols + col0 + cc));
-    *reinterpret_cast<uint4*>(&s_in[t][cc]) = v;
+    // asynchronous 16-byte copy straight into shared memory; nothing is read (and zeros are written) beyond the edges
+    const bool inside = row0 + t < rows && col0 + cc < cols;
+    const uint16_t* g = inside ? src + (row0 + t) * cols + col0 + cc : src;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_in[t][cc])), "l"(g), "r"(inside ? 16 : 0) : "memory");
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
 
   // phase 2: thread -> (column pair 2np, 2np+1; token block c).  One 32-bit shared load brings both
@@ -442,8 +456,8 @@ int launch_quantize(const void* in, void* codes, void* scales, int64_t batch, in
     const int64_t blocks = (n_chunks + kQThreads * kQChunksPerThread - 1) / (kQThreads * kQChunksPerThread);
     if (!tile && blocks > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
     if (tile) {
-      if (rows_pad / kTile > 0x7FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
-      dim3 grid((unsigned)(rows_pad / kTile), (unsigned)batch);
+      if (rows_pad / kTile > 0x3FFFFFFF || batch > 65535) return MXATTN_EUNSUPPORTED;
+      dim3 grid((unsigned)(2 * (rows_pad / kTile)), (unsigned)batch);       // the plain tile kernel takes half a tile per CTA
       if (rotate) {
         auto kern = rule == kRuleOcp ? rot::quantize_axis1_rot_tc_kernel<true, 0>
                   : rule == kRuleUos ? rot::quantize_axis1_rot_tc_kernel<true, 1> : rot::quantize_axis1_rot_tc_kernel<true, 2>;

@@ -145,10 +145,12 @@ quantize_nvfp4_axis0_kernel(const uint16_t* __restrict__ in, uint8_t* __restrict
   for (int k = 0; k < (kTile * kTile / 8) / kThreads; ++k) {
     const int chunk = k * kThreads + tid;
     const int t = chunk >> 4, cc = (chunk & 15) << 3;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row0 + t < rows && col0 + cc < cols) v = __ldg(reinterpret_cast<const uint4*>(src + (row0 + t) * cols + col0 + cc));
-    *reinterpret_cast<uint4*>(&s_in[t][cc]) = v;
+    // asynchronous 16-byte copy straight into shared memory; nothing is read (and zeros are written) beyond the edges
+    const bool inside = row0 + t < rows && col0 + cc < cols;
+    const uint16_t* gsrc = inside ? src + (row0 + t) * cols + col0 + cc : src;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_in[t][cc])), "l"(gsrc), "r"(inside ? 16 : 0) : "memory");
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
   {
     const int np = tid & 63, c = tid >> 6;              // column pair, chunk of 32 tokens
