@@ -75,51 +75,75 @@ __global__ void __launch_bounds__(kThreads) tensor_amax_kernel(const uint4* __re
 }
 
 // ------------------------------------------------------------------------------------------
-// Axis 1 (Q, K: blocks of 16 along the row).  A thread owns one 16-byte chunk (8 elements), two lanes a block.
-// grid = (ceil(chunks / (256 * 8)), batch); canonical layout: chunks = rows * cols / 8 per matrix; tile layout
+// Axis 1 (Q, K: blocks of 16 along the row).  The CTA's 1024 chunks of 16 bytes (16 KiB) arrive in shared memory by
+// asynchronous copies (chunk c at position c ^ ((c >> 3) & 7) within its group of eight: copies and reads both touch
+// every bank group once per quarter warp); a thread then owns four consecutive chunks = two blocks: block maxima
+// without shuffles, one division per block, one 16-byte store of codes and one 2-byte store of scales.
+// grid = (ceil(chunks / 1024), batch); canonical layout: chunks = rows * cols / 8 per matrix; tile layout
 // (cols == 128): chunks = rows_pad * 16, rows beyond `rows` read as zero.
+constexpr int kA1ChunksPerCta = kThreads * 4;
 template <bool kTileLayout>
 __global__ void __launch_bounds__(kThreads)
 quantize_nvfp4_axis1_kernel(const uint4* __restrict__ in, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                             const float* __restrict__ amax, float* __restrict__ tensor_scale, int64_t rows, int64_t cols,
                             int64_t rows_pad) {
-  constexpr int kPerThread = 8;
+  __shared__ uint4 s_v[kA1ChunksPerCta];
+  const int tid = threadIdx.x;
   const int64_t b = blockIdx.y;
-  const float g = encode_scale(amax[b]);
-  if (blockIdx.x == 0 && threadIdx.x == 0 && tensor_scale) tensor_scale[b] = __fdiv_rn(1.0f, g);
   const int64_t chunks_per_row = cols / 8;
   const int64_t n_valid = rows * chunks_per_row;                                  // chunks that exist in the input
   const int64_t n_out = (kTileLayout ? rows_pad : rows) * chunks_per_row;         // chunks that are written
   const uint4* src = in + b * n_valid;
-  const int64_t base = (int64_t)blockIdx.x * (kThreads * kPerThread) + threadIdx.x;
-  uint4 v[kPerThread];
+  const int64_t base = (int64_t)blockIdx.x * kA1ChunksPerCta;
+  auto pos = [](int c) { return c ^ ((c >> 3) & 7); };
 #pragma unroll
-  for (int u = 0; u < kPerThread; ++u) {
-    const int64_t i = base + u * kThreads;
-    v[u] = i < n_valid ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+  for (int u = 0; u < 4; ++u) {
+    const int c = u * kThreads + tid;
+    const bool inside = base + c < n_valid;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(&s_v[pos(c)])),
+                 "l"(inside ? src + base + c : in), "r"(inside ? 16 : 0) : "memory");
   }
+  const float g = encode_scale(amax[b]);
+  if (blockIdx.x == 0 && tid == 0 && tensor_scale) tensor_scale[b] = __fdiv_rn(1.0f, g);
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  const int64_t i = base + 4 * tid;                 // first of this thread's four chunks (n_out is even: whole blocks only)
+  if (i >= n_out) return;
+  uint4 v[4];
 #pragma unroll
-  for (int u = 0; u < kPerThread; ++u) {
-    const int64_t i = base + u * kThreads;
-    uint32_t m = absmax_bf16x8(v[u]);
-    m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-    uint32_t sc;
-    const float r = block_scale(__uint_as_float(m << 16), g, &sc);
-    const uint32_t packed = quantize_bf16x8(v[u], r);
-    if (i >= n_out) continue;
-    if (kTileLayout) {
-      const int64_t row = i >> 4;
-      const int c16 = (int)(i & 15);                   // chunk within the row; block of 16 = c16 / 2, block of 32 = c16 / 4
-      const int64_t tile = b * (rows_pad / kTile) + row / kTile;
-      const int rr = (int)(row % kTile);
-      reinterpret_cast<uint32_t*>(codes + tile * kTileCodeBytes)[tile_code_offset(rr, c16 >> 2) / 4 + (c16 & 3)] = packed;
-      if ((c16 & 1) == 0) {
-        const int blk = c16 >> 1;                      // 0..7
-        scales[tile * kNvTileScaleBytes + (blk >> 2) * kTileScaleBytes + tile_scale_offset(rr, blk & 3)] = (uint8_t)sc;
-      }
+  for (int k = 0; k < 4; ++k) v[k] = s_v[pos(4 * tid + k)];
+  uint32_t sc[2], w[4];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const uint32_t m = max(absmax_bf16x8(v[2 * h]), absmax_bf16x8(v[2 * h + 1]));
+    const float r = block_scale(__uint_as_float(m << 16), g, &sc[h]);
+    w[2 * h] = quantize_bf16x8(v[2 * h], r);
+    w[2 * h + 1] = quantize_bf16x8(v[2 * h + 1], r);
+  }
+  const bool both = i + 2 < n_out;                  // the matrix may end after this thread's first block
+  if (kTileLayout) {                                // 16 chunks per row: the four chunks are one 32-column group of one row
+    const int64_t row = i >> 4;
+    const int q = (int)(i & 15) >> 2;
+    const int64_t tile = b * (rows_pad / kTile) + row / kTile;
+    const int rr = (int)(row % kTile);
+    *reinterpret_cast<uint4*>(codes + tile * kTileCodeBytes + tile_code_offset(rr, q)) = make_uint4(w[0], w[1], w[2], w[3]);
+    // blocks 2q and 2q + 1 of the row: adjacent bytes of one scale-factor atom
+    *reinterpret_cast<uint16_t*>(scales + tile * kNvTileScaleBytes + (q >> 1) * kTileScaleBytes + tile_scale_offset(rr, (2 * q) & 3)) =
+        (uint16_t)(sc[0] | (sc[1] << 8));
+  } else {
+    uint32_t* cdst = reinterpret_cast<uint32_t*>(codes) + b * n_out + i;
+    uint8_t* sdst = scales + b * (n_out / 2) + (i >> 1);
+    if (both && (((b * n_out) & 3) == 0)) {
+      *reinterpret_cast<uint4*>(cdst) = make_uint4(w[0], w[1], w[2], w[3]);
     } else {
-      reinterpret_cast<uint32_t*>(codes)[b * n_out + i] = packed;
-      if ((i & 1) == 0) scales[b * (n_out / 2) + (i >> 1)] = (uint8_t)sc;
+      *reinterpret_cast<uint2*>(cdst) = make_uint2(w[0], w[1]);
+      if (both) *reinterpret_cast<uint2*>(cdst + 2) = make_uint2(w[2], w[3]);
+    }
+    if (both && (((b * (n_out / 2)) & 1) == 0)) {
+      *reinterpret_cast<uint16_t*>(sdst) = (uint16_t)(sc[0] | (sc[1] << 8));
+    } else {
+      sdst[0] = (uint8_t)sc[0];
+      if (both) sdst[1] = (uint8_t)sc[1];
     }
   }
 }
@@ -245,7 +269,7 @@ int launch_quantize_nvfp4(const void* in, void* codes, void* scales, const float
   const bool tile = (layout == MXATTN_LAYOUT_TILE);
   if (block_axis == 1) {
     const int64_t n_out = (tile ? rows_pad : rows) * (cols / 8);
-    const int64_t blocks = (n_out + nv::kThreads * 8 - 1) / (nv::kThreads * 8);
+    const int64_t blocks = (n_out + nv::kA1ChunksPerCta - 1) / nv::kA1ChunksPerCta;
     if (blocks > 0x7FFFFFFF) return MXATTN_EUNSUPPORTED;
     dim3 grid((unsigned)blocks, (unsigned)batch);
     if (tile)
