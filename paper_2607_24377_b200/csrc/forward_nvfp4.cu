@@ -11,10 +11,11 @@
 // is known to be 1); under PNQ l = l_raw * s_T(P) and s_T(P) cancels.
 //
 // Per KV tile a softmax thread (two threads per query row, 64 key columns = 4 blocks of 16 each):
-//   p_i  = exp2(s_i * c - m_new * c)                       one fma + one ex2 per element
-//   per block: M = its largest p (evaluated by the same expression), d = E4M3(fl32(fl32(M * 2688) * fl32(1/6))),
-//              r = fl32(2688 / d)  (0 if d = 0),  codes = E2M1(fl32(p_i * r)),  scale byte = d
-// which is the library's NVFP4 recipe (include/mxattn.h) with the tensor maximum 1.
+//   per block: M = its largest p = exp2(s_max * c - m_new * c), d = E4M3(fl32(fl32(M * 2688) * fl32(1/6))), scale byte = d
+//   per element: codes = E2M1(exp2(s_i * c - m_new * c + log2(2688 / d)))      half a packed fma + one ex2
+// which is the library's NVFP4 recipe (include/mxattn.h) with the tensor maximum 1, the element multiplier
+// r = 2688 / d folded into the exponent (the recipe's fl32(p_i * r) differs from this by about 2e-7 relative, the order
+// of ex2.approx itself; a block with d = 0 keeps r = 1, its codes are 0 either way).
 //
 // One CTA per work item (two query tiles of one head); outputs are stored from registers.  Tensor-memory map:
 // S [0,128), O_0 [128,272), O_1 [272,416), scale factors from 416 (8 columns per operand tile: two atoms).
@@ -61,6 +62,8 @@ constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK
 
 constexpr float kTensorRangeP = 2688.0f;                   // 448 * 6: encode scale of the softmax tile (tensor maximum 1)
 constexpr float kOneSixth = 0.16666667163372040f;          // fl32(1/6)
+constexpr float kLog2TensorRangeP = 11.392317422778762f;   // log2(2688)
+constexpr float kInvTensorRangeP = 3.7202381e-4f;          // fl32(1/2688)
 
 struct Params {
   const uint8_t* q_codes; const uint8_t* q_scales;
@@ -327,8 +330,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_nvfp4_kernel(const Para
       tc_fence_after();
       const bool rescale = __any_sync(0xFFFFFFFFu, moved);
       float alpha = 1.0f;
-      // block scales: the block's largest probability by the elements' own expression, then the two-level recipe
-      float rb[4];
+      // block scales: the block's largest probability by the elements' own expression, then the two-level recipe.
+      // The element multiplier 2688 / d_b is folded into the exponent as its logarithm (one lg2.approx per block in
+      // place of a division per block and a multiply per element; relative difference about 2e-7, the order of
+      // ex2.approx itself).  A block whose scale rounds to zero keeps multiplier 1: its probabilities are below
+      // 2.2e-6 and round to code 0 either way, and the direct placement still sums them.
+      float nb[4], inv_r[4];
       uint32_t sf4 = 0;
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
@@ -336,11 +343,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_nvfp4_kernel(const Para
         const float y = __fmul_rn(__fmul_rn(pm, kTensorRangeP), kOneSixth);
         const uint32_t code = e4m3_encode(y);
         const float d = e4m3_decode(code);
-        rb[b] = d == 0.0f ? 0.0f : __fdiv_rn(kTensorRangeP, d);
+        float lg;
+        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(d));
+        nb[b] = d == 0.0f ? nmc : nmc + (kLog2TensorRangeP - lg);
+        inv_r[b] = d == 0.0f ? 1.0f : d * kInvTensorRangeP;
         sf4 |= code << (8 * b);
       }
       asm volatile("st.shared.b32 [%0], %1;" ::"r"(aSF), "r"(sf4) : "memory");
       float l_tile = 0.0f;
+      const uint64_t cc2 = dup2(c);
       auto tile_body = [&](auto resc_tag) {
         constexpr bool kResc = decltype(resc_tag)::value;
         if (kResc) alpha = ex2((m_old - m_new) * c);
@@ -352,16 +363,15 @@ __global__ void __launch_bounds__(kThreads, 1) attention_nvfp4_kernel(const Para
             uint32_t oc[8];
             const uint32_t t_oc = t_o + kCols * h + 32 * b32 + 8 * g;
             if (kResc) TMEM_LD8(t_oc, oc);
-            const float r = rb[2 * b32 + (g >> 1)];
+            const uint64_t nb2 = dup2(nb[2 * b32 + (g >> 1)]);
             float x[8];
-            float sx = 0.0f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float pv = ex2(fmaf(__uint_as_float(sr[32 * b32 + 8 * g + i]), c, nmc));
-              if (!kPnq) sx += pv;
-              x[i] = __fmul_rn(pv, r);
+            for (int i = 0; i < 8; i += 2) {           // x = exp2(s * c + nb) = p~ * 2688 / d_b, two elements per multiply-add
+              fma2(sr[32 * b32 + 8 * g + i], sr[32 * b32 + 8 * g + i + 1], cc2, nb2, x[i], x[i + 1]);
+              x[i] = ex2(x[i]);
+              x[i + 1] = ex2(x[i + 1]);
             }
-            if (!kPnq) l_tile += sx;
+            if (!kPnq) l_tile = fmaf(((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7])), inv_r[2 * b32 + (g >> 1)], l_tile);
             const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
             if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
             if (kResc) {
