@@ -600,7 +600,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const Params p, 
             }
             const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
             if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
-            if (!kPnq) sx += ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
+            if (!kPnq) {                              // two packed additions and three plain ones per eight elements
+              float s0, s1;
+              add2x2(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7], s0, s1);
+              sx += s0 + s1;
+            }
             if (kResc) {
               tmem_ld_wait();
 #pragma unroll

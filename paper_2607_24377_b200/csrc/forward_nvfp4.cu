@@ -371,7 +371,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_nvfp4_kernel(const Para
               x[i] = ex2(x[i]);
               x[i + 1] = ex2(x[i + 1]);
             }
-            if (!kPnq) l_tile = fmaf(((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7])), inv_r[2 * b32 + (g >> 1)], l_tile);
+            if (!kPnq) {
+              float s0, s1;
+              add2x2(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7], s0, s1);
+              l_tile = fmaf(s0 + s1, inv_r[2 * b32 + (g >> 1)], l_tile);
+            }
             const uint32_t pk = pack_e2m1x8(x[0], x[1], x[2], x[3], x[4], x[5], x[6], x[7]);
             if (g == 0) w.x = pk; else if (g == 1) w.y = pk; else if (g == 2) w.z = pk; else w.w = pk;
             if (kResc) {

@@ -47,6 +47,19 @@ __device__ __forceinline__ void fma2(uint32_t a0_bits, uint32_t a1_bits, uint64_
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(ab), "l"(cc), "l"(dd));
   asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(r));
 }
+// (a0 + a2) + (a4 + a6) and (a1 + a3) + (a5 + a7) with three packed fp32x2 additions (each half an IEEE fp32 add)
+__device__ __forceinline__ void add2x2(float a0, float a1, float a2, float a3, float a4, float a5, float a6, float a7,
+                                       float& r0, float& r1) {
+  uint64_t p0, p1, p2, p3, q0, q1, r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(p0) : "f"(a0), "f"(a1));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(p1) : "f"(a2), "f"(a3));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "f"(a4), "f"(a5));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(p3) : "f"(a6), "f"(a7));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(q0) : "l"(p0), "l"(p1));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(q1) : "l"(p2), "l"(p3));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(q0), "l"(q1));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(r));
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
