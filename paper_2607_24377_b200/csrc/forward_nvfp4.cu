@@ -62,7 +62,6 @@ constexpr uint32_t kColS = 0, kColO0 = 128, kColO1 = 272, kColSFQ = 416, kColSFK
 
 constexpr float kTensorRangeP = 2688.0f;                   // 448 * 6: encode scale of the softmax tile (tensor maximum 1)
 constexpr float kOneSixth = 0.16666667163372040f;          // fl32(1/6)
-constexpr float kLog2TensorRangeP = 11.392317422778762f;   // log2(2688)
 constexpr float kInvTensorRangeP = 3.7202381e-4f;          // fl32(1/2688)
 
 struct Params {
@@ -343,9 +342,16 @@ __global__ void __launch_bounds__(kThreads, 1) attention_nvfp4_kernel(const Para
         const float y = __fmul_rn(__fmul_rn(pm, kTensorRangeP), kOneSixth);
         const uint32_t code = e4m3_encode(y);
         const float d = e4m3_decode(code);
-        float lg;
-        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(d));
-        nb[b] = d == 0.0f ? nmc : nmc + (kLog2TensorRangeP - lg);
+        // log2(2688 / d) from the code's fields: d = (1 + k/8) 2^(E-7), so only the mantissa's logarithm is approximated,
+        // on an argument in [1, 2) where lg2.approx is good to 2^-22 absolute (on d itself its error is relative to
+        // log2 d, about 2e-6 for the blocks that matter, which moves codes across rounding boundaries); the integer part
+        // and log2(2688) = 11 + 0.39231742 are added exactly enough that the sum rounds once at its own magnitude
+        const uint32_t fe = code >> 3, fk = code & 7u;
+        float lgm;
+        asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lgm) : "f"(fe ? __uint_as_float(0x3F800000u | (fk << 20)) : d * 512.0f));
+        const float fef = __uint_as_float(0x4B400000u + fe) - 12582912.0f;           // (float)E without a conversion instruction
+        const float lr = (fe ? 18.0f - fef : 20.0f) + (0.39231742f - lgm);           // subnormal d = k 2^-9
+        nb[b] = d == 0.0f ? nmc : fmaf(-m_new, c, lr);     // one rounding: -(m_new c) + log2(2688 / d)
         inv_r[b] = d == 0.0f ? 1.0f : d * kInvTensorRangeP;
         sf4 |= code << (8 * b);
       }
