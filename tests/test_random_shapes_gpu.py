@@ -122,3 +122,30 @@ def test_random_forward_cases_nvfp4():
         rel = np.linalg.norm(got - want) / np.linalg.norm(want)
         rows_off = int((np.abs(got - want).max(axis=-1) > 4e-3).sum())
         assert rel <= 2.5e-3 and rows_off <= 2, (cfg, pnq, rel, rows_off)
+
+
+def test_random_host_buffer_cases_equal_the_device_path():
+    # mxattn_forward_host pipelines stages of one or more heads over several streams: whatever the number of heads,
+    # the lengths and the flags, its result is the device path's, bit for bit, also when the arena is used twice in a row
+    import paper_2607_24377_b200 as mx
+    rng = np.random.default_rng(41)
+    for _ in range(30):
+        B = int(rng.integers(1, 3)); H = int(rng.integers(1, 41))
+        Nq = int(rng.integers(1, 1200)); Nkv = int(rng.integers(1, 1200))
+        uos, pnq, rot, f32 = bool(rng.integers(2)), bool(rng.integers(2)), bool(rng.random() < 0.3), bool(rng.integers(2))
+        cfg = si.custom_config("rndh", B, H, Nq, Nkv, int(rng.integers(1 << 30)))
+        q, k, v = si.make_all(cfg)
+        flags = (mx.FLAG_UOS if uos else 0) | (mx.FLAG_PNQ if pnq else 0) | (mx.FLAG_HADAMARD if rot else 0) | (mx.FLAG_OUT_FP32 if f32 else 0)
+        dt, bits = (torch.float32, torch.int32) if f32 else (torch.bfloat16, torch.int16)
+        out = torch.full((B, H, Nq, 128), float("nan"), dtype=dt, device="cuda")
+        ws = torch.empty(mx.forward_workspace_bytes(B, H, Nq, Nkv, 128), dtype=torch.uint8, device="cuda")
+        mx.forward_ws(util.to_dev_bf16(q), util.to_dev_bf16(k), util.to_dev_bf16(v), out, B, H, Nq, Nkv, 128, cfg.softmax_scale, flags, ws)
+        assert mx.device_status(ws) == 0
+        want = out.cpu()
+        hq, hk, hv = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (q, k, v))
+        ho = torch.empty((B, H, Nq, 128), dtype=dt).pin_memory()
+        arena = torch.empty(mx.forward_host_arena_bytes(B, H, Nq, Nkv, 128, flags), dtype=torch.uint8, device="cuda")
+        for _rep in range(2):
+            ho.fill_(float("nan"))
+            mx.forward_host(hq, hk, hv, ho, B, H, Nq, Nkv, 128, cfg.softmax_scale, flags, arena)
+            assert torch.equal(ho.view(bits), want.view(bits)), (B, H, Nq, Nkv, uos, pnq, rot, f32)
