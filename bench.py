@@ -474,7 +474,7 @@ def main():
                 # the softmax exponentials bind before the tensor pipe does: 16 ex2 per clock per SM,
                 # one per (query, key) pair, 512 tensor flops per pair
                 "mufu_ceiling_tflops": mufu_ceiling, "frac_of_mufu_ceiling": attn_tflops / mufu_ceiling if mufu_ceiling else None,
-                "ncu_cross_check": "profiles/attention_kernel_sweep16384.txt: sm__pipe_tensor_cycles_active 20.9 %, XU pipe 82 %"}
+                "ncu_cross_check": "profiles/attention_kernel_sweep16384.txt: sm__pipe_tensor_cycles_active 21.2 %, XU pipe 83 %"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
