@@ -4,8 +4,18 @@
 #include <vector>
 
 #include "common.cuh"
+#include <nvtx3/nvToolsExt.h>      // header-only: the ranges cost nothing unless a profiling tool is attached
 
 namespace mxattn {
+
+// NVTX range for the lifetime of the object: the host-side enqueue of a launch or of a pipeline stage, so that a
+// timeline shows which call and which stage queued which kernels.
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 static int g_launches = 0;
 static void* g_workspace = nullptr;
@@ -61,13 +71,17 @@ static int forward_ws(const void* q, const void* k, const void* v, void* o, int 
   if (cudaMemsetAsync(ws + w.status, 0, 16, qs) != cudaSuccess) return MXATTN_ECUDA;
   int rc;
   // Algorithm 2 lines 3-5: Q-hat, K-hat (blocks along d), V-hat (blocks along tokens)
-  if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
-  if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
-  if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+  {
+    TraceRange tr("mxattn quantize Q K V");
+    if ((rc = launch_quantize(q, ws + w.q_codes, ws + w.q_scales, bh, Nq, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+    if ((rc = launch_quantize(k, ws + w.k_codes, ws + w.k_scales, bh, Nkv, d, 1, qk_mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+    if ((rc = launch_quantize(v, ws + w.v_codes, ws + w.v_scales, bh, Nkv, d, 0, mode, MXATTN_LAYOUT_TILE, qs))) return rc;
+  }
   if (qstream) {
     if (cudaEventRecord(qdone, qstream) != cudaSuccess || cudaStreamWaitEvent(stream, qdone, 0) != cudaSuccess) return MXATTN_ECUDA;
   }
   // lines 6-19
+  TraceRange tr("mxattn attention");
   return launch_forward(ws + w.q_codes, ws + w.q_scales, ws + w.k_codes, ws + w.k_scales, ws + w.v_codes,
                         ws + w.v_scales, o, B, H, Nq, Nkv, softmax_scale, flags,
                         reinterpret_cast<int*>(ws + w.status), stream, dump, profile);
@@ -293,6 +307,7 @@ extern "C" int mxattn_forward_host(const void* q_host, const void* k_host, const
   ck(cudaStreamWaitEvent(hp->attn, ev[3 * stages], 0));
   int rc = MXATTN_OK;
   for (size_t st = 0; st < stages && !fail && rc == MXATTN_OK; ++st) {
+    TraceRange tr("mxattn host stage");
     const size_t i = first_head(st), n = first_head(st + 1) - i;  // heads of the stage; heads are contiguous in memory
     // attention launches alternate between the caller's stream and one of the pipeline's, so that the CTAs of a
     // stage start on the SMs the previous stage's last CTAs leave (no tail, no launch gap between stages)
